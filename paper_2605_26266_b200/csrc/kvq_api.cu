@@ -1,0 +1,172 @@
+// C-ABI entry points of libkvq: argument validation and dispatch to the kernels.
+#include "kvq_common.cuh"
+
+namespace kvq {
+
+static thread_local int g_last_cuda_error = 0;
+
+int record_cuda_error(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return KVQ_ERR_CUDA;
+}
+
+int check_shape(const kvq_cache_desc* d) {
+  if (!d) return KVQ_ERR_INVALID_ARG;
+  if (d->batch <= 0 || d->heads <= 0 || d->head_dim <= 0 || d->group <= 0 || d->capacity <= 0)
+    return KVQ_ERR_INVALID_ARG;
+  if (d->head_dim % d->group != 0) return KVQ_ERR_INVALID_ARG;
+  if (d->head_dim != 64 && d->head_dim != 128) return KVQ_ERR_UNSUPPORTED;
+  if (d->bits != 2 && d->bits != 4) return KVQ_ERR_UNSUPPORTED;
+  if (d->group != 32 && d->group != 64 && d->group != 128) return KVQ_ERR_UNSUPPORTED;
+  if (d->capacity % 128 != 0) return KVQ_ERR_INVALID_ARG;
+  return KVQ_OK;
+}
+
+int check_desc(const kvq_cache_desc* d) {
+  int r = check_shape(d);
+  if (r != KVQ_OK) return r;
+  const void* ptrs[6] = {d->k_codes, d->v_codes, d->k_scale, d->v_scale, d->k_zero, d->v_zero};
+  for (const void* p : ptrs) {
+    if (!p) return KVQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return KVQ_ERR_ALIGNMENT;
+  }
+  return KVQ_OK;
+}
+
+int check_tensor(const void* p, kvq_strides s) {
+  if (!p) return KVQ_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return KVQ_ERR_ALIGNMENT;
+  if (s.b < 0 || s.h < 0 || s.t <= 0) return KVQ_ERR_INVALID_ARG;
+  if (s.b % 8 != 0 || s.h % 8 != 0 || s.t % 8 != 0) return KVQ_ERR_ALIGNMENT;
+  return KVQ_OK;
+}
+
+static int check_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t cache_len,
+                           int64_t m_tokens, int64_t n_cur, uint32_t flags) {
+  int r = check_shape(d);
+  if (r != KVQ_OK) return r;
+  if (cache_begin < 0 || cache_len < 0 || m_tokens < 0 || n_cur < 1) return KVQ_ERR_INVALID_ARG;
+  if (cache_begin % 16 != 0) return KVQ_ERR_ALIGNMENT;
+  if (cache_begin + cache_len > d->capacity) return KVQ_ERR_CAPACITY;
+  if (m_tokens > 0x7FFFFFFFLL || n_cur > 0x7FFFFFFFLL || cache_len > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  const uint32_t kern = flags & KVQ_KERNEL_MASK;
+  if (kern != KVQ_KERNEL_AUTO && kern != KVQ_KERNEL_MMA_SYNC && kern != KVQ_KERNEL_TCGEN05)
+    return KVQ_ERR_INVALID_ARG;
+  if (flags & ~(KVQ_CORRECTION_ON | KVQ_KERNEL_MASK)) return KVQ_ERR_INVALID_ARG;
+  return KVQ_OK;
+}
+
+static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur, uint32_t flags, int* err) {
+  const uint32_t kern = flags & KVQ_KERNEL_MASK;
+  *err = KVQ_OK;
+  if (kern == KVQ_KERNEL_MMA_SYNC) return false;
+  const bool ok = attn_tcgen05_supports(d, m_tokens, n_cur);
+  if (kern == KVQ_KERNEL_TCGEN05 && !ok) *err = KVQ_ERR_UNSUPPORTED;
+  return ok;
+}
+
+}  // namespace kvq
+
+using namespace kvq;
+
+extern "C" {
+
+int kvq_version(void) { return KVQ_VERSION; }
+
+int kvq_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* kvq_status_string(int status) {
+  switch (status) {
+    case KVQ_OK: return "ok";
+    case KVQ_ERR_INVALID_ARG: return "invalid argument";
+    case KVQ_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case KVQ_ERR_ALIGNMENT: return "pointer or stride alignment";
+    case KVQ_ERR_CAPACITY: return "cache capacity exceeded";
+    case KVQ_ERR_CUDA: return "CUDA error";
+    case KVQ_ERR_TIMEOUT: return "device-side wait timed out";
+    case KVQ_ERR_WORKSPACE: return "workspace missing or too small";
+    default: return "unknown status";
+  }
+}
+
+int kvq_cache_bytes(const kvq_cache_desc* desc, size_t out_bytes[6]) {
+  int r = check_shape(desc);
+  if (r != KVQ_OK) return r;
+  if (!out_bytes) return KVQ_ERR_INVALID_ARG;
+  const size_t tok = (size_t)desc->batch * desc->heads * (size_t)desc->capacity;
+  const size_t G = (size_t)groups_of(desc);
+  out_bytes[0] = out_bytes[1] = tok * (size_t)code_bytes_of(desc);
+  out_bytes[2] = out_bytes[3] = tok * G;
+  out_bytes[4] = out_bytes[5] = tok * G * 2;
+  return KVQ_OK;
+}
+
+int kvq_quantize_append(const kvq_cache_desc* desc, int64_t cache_len, const void* k_bf16,
+                        const void* v_bf16, kvq_strides kv, int64_t n_tokens, kvq_stream_t stream) {
+  int r = check_desc(desc);
+  if (r != KVQ_OK) return r;
+  if (cache_len < 0 || n_tokens < 0) return KVQ_ERR_INVALID_ARG;
+  if (cache_len + n_tokens > desc->capacity) return KVQ_ERR_CAPACITY;
+  if ((r = check_tensor(k_bf16, kv)) != KVQ_OK) return r;
+  if ((r = check_tensor(v_bf16, kv)) != KVQ_OK) return r;
+  if (n_tokens == 0) return KVQ_OK;
+  return launch_quantize_append(desc, cache_len, k_bf16, v_bf16, kv, n_tokens, (cudaStream_t)stream);
+}
+
+int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len, int64_t m_tokens,
+                             int64_t n_cur, uint32_t flags, size_t* out_bytes) {
+  if (!out_bytes) return KVQ_ERR_INVALID_ARG;
+  int r = check_attn_args(desc, 0, cache_len, m_tokens, n_cur, flags);
+  if (r != KVQ_OK) return r;
+  int err;
+  const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
+  if (err != KVQ_OK) return err;
+  *out_bytes = tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0;
+  return KVQ_OK;
+}
+
+int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
+                       const void* q, kvq_strides q_strides, const void* k_cur, const void* v_cur,
+                       kvq_strides kv_strides, int64_t m_tokens, int64_t n_cur, void* out_bf16,
+                       kvq_strides o_strides, float softmax_scale, uint32_t flags, float* lse_out,
+                       float* cached_mass_out, void* workspace, size_t workspace_bytes,
+                       int32_t* status_word, kvq_stream_t stream) {
+  int r = check_attn_args(desc, cache_begin, cache_len, m_tokens, n_cur, flags);
+  if (r != KVQ_OK) return r;
+  if ((r = check_desc(desc)) != KVQ_OK) return r;
+  if ((r = check_tensor(q, q_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(k_cur, kv_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
+  int err;
+  const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
+  if (err != KVQ_OK) return err;
+  if (tc) {
+    const size_t need = attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur);
+    if (need > 0) {
+      if (!workspace || workspace_bytes < need) return KVQ_ERR_WORKSPACE;
+      if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return KVQ_ERR_ALIGNMENT;
+    }
+  }
+  if (m_tokens == 0) return KVQ_OK;
+  AttnArgs a;
+  a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;
+  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides;
+  a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out_bf16; a.os = o_strides;
+  a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse_out; a.cached_mass = cached_mass_out;
+  a.workspace = workspace; a.workspace_bytes = workspace_bytes; a.status_word = status_word;
+  a.stream = (cudaStream_t)stream;
+  return tc ? launch_attn_tcgen05(a) : launch_attn_mma_sync(a);
+}
+
+int kvq_unpack_codes(const kvq_cache_desc* desc, int which, int64_t begin, int64_t n,
+                     uint8_t* out_codes, kvq_stream_t stream) {
+  int r = check_desc(desc);
+  if (r != KVQ_OK) return r;
+  if ((which != 0 && which != 1) || begin < 0 || n < 0 || !out_codes) return KVQ_ERR_INVALID_ARG;
+  if (begin + n > desc->capacity) return KVQ_ERR_CAPACITY;
+  return launch_unpack_codes(desc, which, begin, n, out_codes, (cudaStream_t)stream);
+}
+
+}  // extern "C"

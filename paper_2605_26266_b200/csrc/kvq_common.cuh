@@ -1,0 +1,81 @@
+// Shared host/device helpers of libkvq (internal; not part of the C ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvq.h"
+
+namespace kvq {
+
+// Records a failing CUDA runtime call for kvq_last_cuda_error() and maps it to KVQ_ERR_CUDA.
+int record_cuda_error(cudaError_t e);
+
+#define KVQ_CUDA_TRY(expr)                                   \
+  do {                                                       \
+    cudaError_t kvq_e_ = (expr);                             \
+    if (kvq_e_ != cudaSuccess) return ::kvq::record_cuda_error(kvq_e_); \
+  } while (0)
+
+// Shape part of the descriptor check (no pointers).
+int check_shape(const kvq_cache_desc* d);
+// Shape + the six buffer pointers.
+int check_desc(const kvq_cache_desc* d);
+int check_tensor(const void* p, kvq_strides s);
+
+inline int groups_of(const kvq_cache_desc* d) { return d->head_dim / d->group; }
+inline int code_bytes_of(const kvq_cache_desc* d) { return d->head_dim * d->bits / 8; }
+
+// launchers implemented in the kernel translation units
+int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const void* k, const void* v,
+                           kvq_strides kv, int64_t n_tokens, cudaStream_t st);
+int launch_unpack_codes(const kvq_cache_desc* d, int which, int64_t begin, int64_t n, uint8_t* out,
+                        cudaStream_t st);
+
+struct AttnArgs {
+  const kvq_cache_desc* desc;
+  int64_t cache_begin, cache_len;
+  const void* q; kvq_strides qs;
+  const void* k_cur; const void* v_cur; kvq_strides kvs;
+  int64_t m_tokens, n_cur;
+  void* out; kvq_strides os;
+  float softmax_scale;
+  uint32_t flags;
+  float* lse; float* cached_mass;
+  void* workspace; size_t workspace_bytes;
+  int32_t* status_word;
+  cudaStream_t stream;
+};
+int launch_attn_mma_sync(const AttnArgs& a);
+// tcgen05 kernel: returns KVQ_ERR_UNSUPPORTED for shapes it does not cover.
+bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur);
+size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
+int launch_attn_tcgen05(const AttnArgs& a);
+
+#ifdef __CUDACC__
+// ---- device-side number-format helpers -------------------------------------------------
+
+// FP32 -> E4M3 byte, round-to-nearest-even, saturating to +-448 (hardware conversion).
+__device__ __forceinline__ uint32_t f32_to_e4m3_byte(float x) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.0f), "f"(x));
+  return r & 0xFFu;
+}
+
+// E4M3 byte -> FP32 (exact).
+__device__ __forceinline__ float e4m3_byte_to_f32(uint32_t b) {
+  uint32_t h2;
+  uint16_t in = (uint16_t)(b & 0xFFu);
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(in));
+  __half lo = __ushort_as_half((unsigned short)(h2 & 0xFFFFu));
+  return __half2float(lo);
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
+  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x));
+}
+#endif
+
+}  // namespace kvq

@@ -1,0 +1,242 @@
+// Quantize-append kernel: Hadamard rotation (keys), group-wise asymmetric round-to-nearest
+// quantization (Eq. (1)), bit packing and coalesced append of one finished chunk's K and V.
+//
+// One warp owns one token-head vector at a time: lane l holds channels [l*EPL, (l+1)*EPL)
+// (EPL = head_dim/32).  The Walsh-Hadamard butterfly runs its first log2(EPL) stages inside a
+// lane and the remaining five across lanes with shuffles; group minimum/maximum are shuffle
+// reductions over the lanes of a group.  Every add, subtract, multiply and divide is a single
+// IEEE binary32 operation (no contraction), so the stored codes, steps and zero-points are
+// reproducible bit for bit.  A CTA stages the packed bytes of 32 consecutive tokens in shared
+// memory and writes them out with 128-bit stores (tokens of one (batch, head) are contiguous
+// in the cache).  The kernel is HBM-bound on its BF16 input.
+#include "kvq_common.cuh"
+
+namespace kvq {
+namespace {
+
+constexpr int kTileTokens = 32;
+constexpr int kWarps = 8;
+constexpr int kTokPerWarp = kTileTokens / kWarps;
+
+struct QParams {
+  const uint16_t* k; const uint16_t* v;
+  int64_t sb, sh, st;          // element strides of k and v
+  int64_t n_tokens, cache_len, capacity;
+  int heads, group, rotate;
+  const int8_t* signs;
+  uint8_t* codes[2]; uint8_t* scale[2]; uint16_t* zero[2];
+  int tiles_per_bh;
+};
+
+template <int EPL>
+__device__ __forceinline__ void load_vec(const uint16_t* p, int lane, float (&x)[EPL]) {
+  if constexpr (EPL == 4) {
+    uint2 r = __ldg(reinterpret_cast<const uint2*>(p) + lane);
+    x[0] = bf16_bits_to_f32(r.x & 0xFFFFu); x[1] = bf16_bits_to_f32(r.x >> 16);
+    x[2] = bf16_bits_to_f32(r.y & 0xFFFFu); x[3] = bf16_bits_to_f32(r.y >> 16);
+  } else {
+    uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(p) + lane);
+    x[0] = bf16_bits_to_f32(r & 0xFFFFu); x[1] = bf16_bits_to_f32(r >> 16);
+  }
+}
+
+// y = c_d * H_d * x, stages h = 1, 2, 4, ... in that order, one rounding per operation.
+template <int EPL>
+__device__ __forceinline__ void hadamard(float (&x)[EPL], int lane, float c_d) {
+#pragma unroll
+  for (int h = 1; h < EPL; h *= 2) {
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      if ((i & h) == 0) {
+        float a = x[i], b = x[i + h];
+        x[i] = __fadd_rn(a, b);
+        x[i + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+#pragma unroll
+  for (int lm = 1; lm < 32; lm *= 2) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
+      x[e] = (lane & lm) ? __fsub_rn(o, x[e]) : __fadd_rn(x[e], o);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], c_d);
+}
+
+// Quantizes the vector held by the warp and stages codes / step / zero-point of token slot
+// `tok` in shared memory.
+template <int EPL, int BITS>
+__device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int lane, int group, int tok,
+                                               uint32_t* s_codes, uint8_t* s_scale, uint16_t* s_zero) {
+  constexpr float L = (float)((1 << BITS) - 1);
+  constexpr int kBitsPerLane = EPL * BITS;
+  constexpr int kLanesPerWord = 32 / kBitsPerLane;
+  constexpr int kWordsPerTok = 32 / kLanesPerWord;
+  const int lanes_per_group = group / EPL;
+  const int G = (32 * EPL) / group;
+
+  float mn = x[0], mx = x[0];
+#pragma unroll
+  for (int e = 1; e < EPL; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+  for (int off = 1; off < lanes_per_group; off *= 2) {
+    mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+  }
+  const float step = __fdiv_rn(__fsub_rn(mx, mn), L);
+  uint32_t sbyte = f32_to_e4m3_byte(step);
+  if (sbyte == 0) sbyte = 1;                       // floor at the smallest subnormal 2^-9
+  const float ds = e4m3_byte_to_f32(sbyte);
+  const float z = __fsub_rn(0.0f, rintf(__fdiv_rn(mn, ds)));
+  const uint32_t zbits = f32_to_bf16_bits(z);
+  const float zs = bf16_bits_to_f32(zbits);
+
+  uint32_t piece = 0;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) {
+    float c = __fadd_rn(rintf(__fdiv_rn(x[e], ds)), zs);
+    c = fminf(fmaxf(c, 0.0f), L);
+    piece |= ((uint32_t)c) << (e * BITS);
+  }
+  uint32_t word = piece << ((lane % kLanesPerWord) * kBitsPerLane);
+#pragma unroll
+  for (int off = 1; off < kLanesPerWord; off *= 2) word |= __shfl_xor_sync(0xFFFFFFFFu, word, off);
+  if ((lane % kLanesPerWord) == 0) s_codes[tok * kWordsPerTok + lane / kLanesPerWord] = word;
+  if ((lane % lanes_per_group) == 0) {
+    s_scale[tok * G + lane / lanes_per_group] = (uint8_t)sbyte;
+    s_zero[tok * G + lane / lanes_per_group] = (uint16_t)zbits;
+  }
+}
+
+// Cooperative shared->global copy with the widest store both sides allow.
+__device__ __forceinline__ void copy_out(uint8_t* dst, const uint8_t* src, int nbytes, int tid, int nthreads) {
+  const uintptr_t a = reinterpret_cast<uintptr_t>(dst) | (uintptr_t)nbytes;
+  if ((a & 15) == 0) {
+    for (int i = tid; i < nbytes / 16; i += nthreads)
+      reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+  } else if ((a & 3) == 0) {
+    for (int i = tid; i < nbytes / 4; i += nthreads)
+      reinterpret_cast<uint32_t*>(dst)[i] = reinterpret_cast<const uint32_t*>(src)[i];
+  } else if ((a & 1) == 0) {
+    for (int i = tid; i < nbytes / 2; i += nthreads)
+      reinterpret_cast<uint16_t*>(dst)[i] = reinterpret_cast<const uint16_t*>(src)[i];
+  } else {
+    for (int i = tid; i < nbytes; i += nthreads) dst[i] = src[i];
+  }
+}
+
+template <int D, int BITS>
+__global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p) {
+  constexpr int EPL = D / 32;
+  constexpr int CB = D * BITS / 8;
+  __shared__ __align__(16) uint32_t s_codes[2][kTileTokens * CB / 4];
+  __shared__ __align__(16) uint8_t s_scale[2][kTileTokens * 4];
+  __shared__ __align__(16) uint16_t s_zero[2][kTileTokens * 4];
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int bh = blockIdx.x / p.tiles_per_bh;
+  const int tile = blockIdx.x - bh * p.tiles_per_bh;
+  const int b = bh / p.heads, h = bh - b * p.heads;
+  const int64_t t0 = (int64_t)tile * kTileTokens;
+  const int nt = (int)min((int64_t)kTileTokens, p.n_tokens - t0);
+  const int G = D / p.group;
+  const float c_d = (D == 64) ? 0.125f : __uint_as_float(0x3DB504F3u);
+
+  float sgn[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) sgn[e] = p.signs ? (float)p.signs[lane * EPL + e] : 1.0f;
+
+  const int64_t base = (int64_t)b * p.sb + (int64_t)h * p.sh;
+  float xk[kTokPerWarp][EPL], xv[kTokPerWarp][EPL];
+#pragma unroll
+  for (int i = 0; i < kTokPerWarp; ++i) {
+    const int tok = warp * kTokPerWarp + i;
+    if (tok < nt) {
+      const int64_t off = base + (t0 + tok) * p.st;
+      load_vec<EPL>(p.k + off, lane, xk[i]);
+      load_vec<EPL>(p.v + off, lane, xv[i]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kTokPerWarp; ++i) {
+    const int tok = warp * kTokPerWarp + i;
+    if (tok < nt) {
+      if (p.rotate) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) xk[i][e] *= sgn[e];
+        hadamard<EPL>(xk[i], lane, c_d);
+      }
+      quantize_stage<EPL, BITS>(xk[i], lane, p.group, tok, s_codes[0], s_scale[0], s_zero[0]);
+      quantize_stage<EPL, BITS>(xv[i], lane, p.group, tok, s_codes[1], s_scale[1], s_zero[1]);
+    }
+  }
+  __syncthreads();
+  const int64_t tok_index = (int64_t)bh * p.capacity + p.cache_len + t0;
+#pragma unroll
+  for (int w = 0; w < 2; ++w) {
+    copy_out(p.codes[w] + tok_index * CB, reinterpret_cast<const uint8_t*>(s_codes[w]), nt * CB, threadIdx.x, kWarps * 32);
+    copy_out(p.scale[w] + tok_index * G, s_scale[w], nt * G, threadIdx.x, kWarps * 32);
+    copy_out(reinterpret_cast<uint8_t*>(p.zero[w] + tok_index * G), reinterpret_cast<const uint8_t*>(s_zero[w]),
+             nt * G * 2, threadIdx.x, kWarps * 32);
+  }
+}
+
+template <int BITS>
+__global__ void unpack_codes_kernel(const uint8_t* codes, uint8_t* out, int64_t capacity, int64_t begin,
+                                    int64_t n, int D, int64_t total) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % D);
+  const int64_t t = (i / D) % n;
+  const int64_t bh = i / ((int64_t)D * n);
+  const int CB = D * BITS / 8;
+  const uint8_t byte = codes[(bh * capacity + begin + t) * CB + (c * BITS) / 8];
+  out[i] = (byte >> ((c * BITS) % 8)) & ((1 << BITS) - 1);
+}
+
+}  // namespace
+
+int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const void* k, const void* v,
+                           kvq_strides kv, int64_t n_tokens, cudaStream_t st) {
+  QParams p;
+  p.k = static_cast<const uint16_t*>(k);
+  p.v = static_cast<const uint16_t*>(v);
+  p.sb = kv.b; p.sh = kv.h; p.st = kv.t;
+  p.n_tokens = n_tokens; p.cache_len = cache_len; p.capacity = d->capacity;
+  p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
+  p.signs = d->signs;
+  p.codes[0] = static_cast<uint8_t*>(d->k_codes); p.codes[1] = static_cast<uint8_t*>(d->v_codes);
+  p.scale[0] = static_cast<uint8_t*>(d->k_scale); p.scale[1] = static_cast<uint8_t*>(d->v_scale);
+  p.zero[0] = static_cast<uint16_t*>(d->k_zero); p.zero[1] = static_cast<uint16_t*>(d->v_zero);
+  p.tiles_per_bh = (int)((n_tokens + kTileTokens - 1) / kTileTokens);
+  const int64_t blocks = (int64_t)d->batch * d->heads * p.tiles_per_bh;
+  if (blocks > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  dim3 grid((unsigned)blocks), block(kWarps * 32);
+  if (d->head_dim == 128 && d->bits == 2) quantize_append_kernel<128, 2><<<grid, block, 0, st>>>(p);
+  else if (d->head_dim == 128 && d->bits == 4) quantize_append_kernel<128, 4><<<grid, block, 0, st>>>(p);
+  else if (d->head_dim == 64 && d->bits == 2) quantize_append_kernel<64, 2><<<grid, block, 0, st>>>(p);
+  else if (d->head_dim == 64 && d->bits == 4) quantize_append_kernel<64, 4><<<grid, block, 0, st>>>(p);
+  else return KVQ_ERR_UNSUPPORTED;
+  KVQ_CUDA_TRY(cudaGetLastError());
+  return KVQ_OK;
+}
+
+int launch_unpack_codes(const kvq_cache_desc* d, int which, int64_t begin, int64_t n, uint8_t* out,
+                        cudaStream_t st) {
+  const int64_t total = (int64_t)d->batch * d->heads * n * d->head_dim;
+  if (total == 0) return KVQ_OK;
+  const uint8_t* codes = static_cast<const uint8_t*>(which == 0 ? d->k_codes : d->v_codes);
+  const int threads = 256;
+  const int64_t blocks = (total + threads - 1) / threads;
+  if (blocks > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  if (d->bits == 2)
+    unpack_codes_kernel<2><<<(unsigned)blocks, threads, 0, st>>>(codes, out, d->capacity, begin, n, d->head_dim, total);
+  else
+    unpack_codes_kernel<4><<<(unsigned)blocks, threads, 0, st>>>(codes, out, d->capacity, begin, n, d->head_dim, total);
+  KVQ_CUDA_TRY(cudaGetLastError());
+  return KVQ_OK;
+}
+
+}  // namespace kvq

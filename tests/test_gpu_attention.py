@@ -1,0 +1,181 @@
+"""GPU parity: kvq_attn_corrected against the oracle (Algorithm 1 in FP64), through the C ABI.
+Tolerances: relative L2 <= 1e-2 and max-abs <= 2e-2 on the BF16 output."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import kvq_oracle as O
+from paper_2605_26266_b200 import inputs
+from tests import kvq_testlib as T
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2605_26266_b200 import binding
+    return binding
+
+
+def kernels(B):
+    return [("auto", B.KVQ_KERNEL_AUTO), ("mma_sync", B.KVQ_KERNEL_MMA_SYNC)]
+
+
+def _build(B, w, chunks, tokens=None, rotate=True, signs=None, units=None, cap=None):
+    """GPU cache of all heads; oracle cache of `units` (or all heads); returns also the current chunk."""
+    cap = cap or w.capacity
+    g = B.Cache(w.batch, w.heads, w.head_dim, w.bits, w.group, cap, rotate_k=rotate, signs=signs)
+    nu = (w.batch, w.heads) if units is None else (1, len(units))
+    o = O.Cache(nu[0], nu[1], w.head_dim, w.bits, w.group, cap, rotate_k=rotate, signs=signs)
+    sel = (lambda a: a) if units is None else (lambda a: np.stack([a[b, h] for (b, h) in units])[None])
+    n = 0
+    for c in range(chunks):
+        _, k, v = inputs.make_chunk(w, c, tokens=tokens)
+        B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
+        n = O.quantize_append(o, n, sel(k), sel(v))
+    return g, o, n, sel
+
+
+def _compare(B, g, o, n_cache, q, kc, vc, sigma, sel, rows=None, flags_list=None, begin=0, check_aux=True):
+    qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+    res = {}
+    for corr in (True, False):
+        want = O.attn_corrected(o, begin, n_cache, sel(q), sel(kc), sel(vc), sigma, correction=corr, rows=rows)
+        for kname, kflag in (flags_list or kernels(B)):
+            flags = (B.KVQ_CORRECTION_ON if corr else B.KVQ_CORRECTION_OFF) | kflag
+            lse = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
+            mass = torch.zeros_like(lse)
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            out = B.kvq_attn_corrected(g, qd, kd, vd, sigma, flags, cache_begin=begin, cache_len=n_cache,
+                                       lse=lse, cached_mass=mass, status_word=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            got = sel(T.from_dev_bf16(out))[0]
+            lse_g = sel(lse.cpu().numpy().astype(np.float64))[0]
+            mass_g = sel(mass.cpu().numpy().astype(np.float64))[0]
+            if rows is not None:
+                got, lse_g, mass_g = got[:, rows], lse_g[:, rows], mass_g[:, rows]
+            res[(corr, kname)] = T.assert_attn_close(got, want["out"], f"corr={corr} kernel={kname}")
+            if check_aux:
+                assert np.abs(lse_g - want["lse"]).max() < 2e-2, kname
+                assert np.abs(mass_g - want["cached_mass"]).max() < 1e-2, kname
+    return res
+
+
+def test_tiny_config_full_parity(B):
+    w = inputs.WORKLOADS["tiny"]
+    g, o, n, sel = _build(B, w, w.cached_chunks)
+    q, kc, vc = inputs.make_chunk(w, w.cached_chunks)
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(w.head_dim), sel)
+
+
+@pytest.mark.parametrize("d,bits,group", [(64, 2, 32), (64, 4, 64), (128, 2, 32), (128, 2, 64),
+                                          (128, 2, 128), (128, 4, 32), (128, 4, 128)])
+def test_ragged_shapes_all_formats(B, d, bits, group):
+    # m, cache and current lengths that are no multiple of any tile size
+    w = inputs.Workload("rag", 200 + d + bits + group, 2, 3, d, 173, 0, bits, group, 3,
+                        k_outliers=2, k_outlier_scale=6.0, head_scale=True)
+    signs = np.random.default_rng(group).choice([-1, 1], size=d).astype(np.int8)
+    g, o, n, sel = _build(B, w, 3, tokens=111, signs=signs, cap=512)
+    assert n == 333
+    q, _, _ = inputs.make_chunk(w, 5, tokens=173)
+    _, kc, vc = inputs.make_chunk(w, 6, tokens=77)
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(d), sel)
+
+
+def test_empty_cache_is_plain_attention(B):
+    w = inputs.Workload("empty", 300, 1, 2, 128, 150, 0, 2, 64, 0)
+    g = B.Cache(1, 2, 128, 2, 64, 128)
+    o = O.Cache(1, 2, 128, 2, 64, 128)
+    q, kc, vc = inputs.make_chunk(w, 0)
+    res = _compare(B, g, o, 0, q, kc, vc, T.sigma_of(128), lambda a: a)
+    # library attention in BF16 on the same device agrees too
+    qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+    ref = torch.nn.functional.scaled_dot_product_attention(qd.float(), kd.float(), vd.float())
+    out = B.kvq_attn_corrected(g, qd, kd, vd, T.sigma_of(128), B.KVQ_CORRECTION_ON, cache_len=0)
+    assert (out.float() - ref).abs().max().item() < 2e-2
+
+
+def test_zero_steps_make_correction_a_noop(B):
+    w = inputs.Workload("zstep", 301, 1, 2, 128, 96, 0, 2, 32, 0)
+    g, o, n, sel = _build(B, w, 2, tokens=100, cap=256)
+    g.views()["k_scale"].zero_()
+    o.k_scale[:] = 0
+    q, kc, vc = inputs.make_chunk(w, 3)
+    qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+    for _, kflag in kernels(B):
+        on = B.kvq_attn_corrected(g, qd, kd, vd, T.sigma_of(128), B.KVQ_CORRECTION_ON | kflag)
+        off = B.kvq_attn_corrected(g, qd, kd, vd, T.sigma_of(128), B.KVQ_CORRECTION_OFF | kflag)
+        assert torch.equal(on, off) and torch.isfinite(on.float()).all()
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(128), sel)
+
+
+def test_rotation_off_window_scale_and_strides(B):
+    # no rotation (Eq. (15) with the unrotated query), a window inside the cache, a softmax
+    # scale other than 1/sqrt(d), and non-contiguous q/k/v/out
+    w = inputs.Workload("norot", 302, 1, 4, 128, 130, 0, 2, 64, 0, k_outliers=2, k_outlier_scale=4.0)
+    g, o, n, sel = _build(B, w, 2, tokens=120, rotate=False, cap=256)
+    q, kc, vc = inputs.make_chunk(w, 4)
+    sigma = 0.05
+    _compare(B, g, o, 150, q, kc, vc, sigma, sel, begin=48)
+    # strided tensors: [B, n, H, d] storage viewed as [B, H, n, d]
+    qd, kd, vd = [T.to_dev(a).permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for a in (q, kc, vc)]
+    out = torch.empty_like(qd)
+    assert not out.is_contiguous()
+    B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON, cache_begin=48, cache_len=150, out=out)
+    want = O.attn_corrected(o, 48, 150, q, kc, vc, sigma, correction=True)["out"]
+    T.assert_attn_close(T.from_dev_bf16(out), want, "strided")
+
+
+def test_correction_lowers_cached_mass_and_mass_is_consistent(B):
+    w = inputs.WORKLOADS["tiny"]
+    g, o, n, sel = _build(B, w, 4)
+    q, kc, vc = inputs.make_chunk(w, 4)
+    qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+    masses = {}
+    for corr in (B.KVQ_CORRECTION_ON, B.KVQ_CORRECTION_OFF):
+        mass = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
+        B.kvq_attn_corrected(g, qd, kd, vd, 0.125, corr, cached_mass=mass)
+        masses[corr] = mass
+    assert (masses[B.KVQ_CORRECTION_ON] < masses[B.KVQ_CORRECTION_OFF]).all()
+    assert (masses[B.KVQ_CORRECTION_OFF] <= 1).all() and (masses[B.KVQ_CORRECTION_ON] > 0).all()
+
+
+@pytest.mark.parametrize("name", ["sweep_int4", "sweep_int2"])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_sweep_config_full_rows(B, name, seed):
+    w = inputs.with_seed(inputs.WORKLOADS[name], seed)
+    units = [(0, 0), (0, 7), (0, 15)] if seed == 0 else [(0, 3)]
+    g, o, n, sel = _build(B, w, w.cached_chunks, units=units)
+    q, kc, vc = inputs.make_chunk(w, w.cached_chunks)
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(w.head_dim), sel)
+
+
+@pytest.mark.parametrize("name,units", [("dit", [(0, 2), (0, 23)]), ("long", [(0, 13)])])
+def test_large_configs_sampled_rows(B, name, units):
+    """Full-size launch; oracle on sampled rows touching every 128-row tile, for a few heads."""
+    w = inputs.WORKLOADS[name]
+    g, o, n, sel = _build(B, w, w.cached_chunks, units=units)
+    q, kc, vc = inputs.make_chunk(w, w.cached_chunks)
+    rows = inputs.sample_rows(w.chunk, 128, 32, seed=w.cfg_id)
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(w.head_dim), sel, rows=rows)
+
+
+def test_pipeline_config_steps(B):
+    """Attend-then-append over successive chunks (steps 0, 1, 2 and 5 checked; step 0 has an empty cache)."""
+    w = inputs.WORKLOADS["pipeline"]
+    units = [(0, 0), (1, 20)]
+    sel = lambda a: np.stack([a[b, h] for (b, h) in units])[None]
+    g = B.Cache(w.batch, w.heads, w.head_dim, w.bits, w.group, w.capacity)
+    o = O.Cache(1, len(units), w.head_dim, w.bits, w.group, w.capacity)
+    rows = inputs.sample_rows(w.chunk, 128, 16, seed=5)
+    n = 0
+    for step in range(6):
+        q, k, v = inputs.make_chunk(w, step)
+        if step in (0, 1, 2, 5):
+            _compare(B, g, o, n, q, k, v, T.sigma_of(w.head_dim), sel, rows=rows)
+        B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
+        n = O.quantize_append(o, n, sel(k), sel(v))
+    T.assert_cache_equal(T.gpu_cache_arrays(g, n), o, n, units=units)
