@@ -5,8 +5,13 @@
 // online softmax: a CTA owns 64 query rows (4 warps x 16 rows), walks the cached keys in
 // tiles of 64 (dequantized on the fly into shared memory, never to HBM), subtracts the
 // Taylor bias from those scores, then walks the current chunk's BF16 keys with the
-// unrotated query and no bias, and normalises once at the end.  The tcgen05 kernel is the
-// fast path for the large shapes; this one is the cross-check and covers everything else.
+// unrotated query and no bias, and normalises once at the end.  The rotated query and the
+// dequantized keys are held in FP16 (11-bit significands; the rotated query is not exactly
+// representable in BF16 and its rounding would dominate the error budget on heavy-tailed
+// keys), so the cached-score contraction is FP16 x FP16 -> FP32; everything else is BF16.
+// Rotated queries and dequantized keys must stay below the FP16 maximum (65504); queries
+// are clamped there.  The tcgen05 kernel is the fast path for the large shapes; this one is
+// the cross-check and covers everything else.
 #include "kvq_common.cuh"
 
 namespace kvq {
@@ -45,8 +50,18 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  lo = fminf(fmaxf(lo, -65504.f), 65504.f);
+  hi = fminf(fmaxf(hi, -65504.f), 65504.f);
+  return (uint32_t)__half_as_ushort(__float2half_rn(lo)) | ((uint32_t)__half_as_ushort(__float2half_rn(hi)) << 16);
 }
 
 template <int D, int BITS>
@@ -71,8 +86,9 @@ __device__ __forceinline__ void load_packed(Packed<D, BITS>& r, const uint8_t* c
   }
 }
 
-// x_hat = (code - zero) * step, rounded once to BF16, written to row `key` of a [kBN][D+8] tile.
-template <int D, int BITS>
+// x_hat = (code - zero) * step, rounded once to FP16 (keys) or BF16 (values), written to row
+// `key` of a [kBN][D+8] tile.
+template <int D, int BITS, bool kHalf>
 __device__ __forceinline__ void dequant_store(const Packed<D, BITS>& r, uint16_t* tile, int key, int half, int group) {
   constexpr int LD = D + 8;
   constexpr int per = 32 / BITS;
@@ -90,7 +106,7 @@ __device__ __forceinline__ void dequant_store(const Packed<D, BITS>& r, uint16_t
       const int c0 = c8 + e, c1 = c8 + e + 1;
       const float x0 = ((float)((r.w[c0 / per] >> ((c0 % per) * BITS)) & mask) - zs) * ds;
       const float x1 = ((float)((r.w[c1 / per] >> ((c1 % per) * BITS)) & mask) - zs) * ds;
-      o[e / 2] = pack_bf16(x0, x1);
+      o[e / 2] = kHalf ? pack_f16(x0, x1) : pack_bf16(x0, x1);
     }
     *reinterpret_cast<uint4*>(row + c8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
@@ -104,7 +120,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
   constexpr int NBO = D / 8;       // n-blocks of the output
   extern __shared__ __align__(16) uint8_t smem_raw[];
   uint16_t* sQ = reinterpret_cast<uint16_t*>(smem_raw);       // unrotated query  [kBM][LD]
-  uint16_t* sQr = sQ + kBM * LD;                               // rotated query    [kBM][LD]
+  uint16_t* sQr = sQ + kBM * LD;                               // rotated query    [kBM][LD], FP16
   uint16_t* sK = sQr + kBM * LD;                               // key tile         [kBN][LD]
   uint16_t* sV = sK + kBN * LD;                                // value tile       [kBN][LD]
   float* sNu = reinterpret_cast<float*>(sV + kBN * LD);        // [kBM][4]
@@ -163,7 +179,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
       if ((lane % lanes_per_group) == 0) sNu[r * 4 + lane / lanes_per_group] = nu;
 #pragma unroll
       for (int e = 0; e < EPL / 2; ++e)
-        reinterpret_cast<uint32_t*>(sQr + r * LD + lane * EPL)[e] = pack_bf16(x[2 * e], x[2 * e + 1]);
+        reinterpret_cast<uint32_t*>(sQr + r * LD + lane * EPL)[e] = pack_f16(x[2 * e], x[2 * e + 1]);
     }
   }
   __syncthreads();
@@ -196,8 +212,13 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
       for (int nb2 = 0; nb2 < kBN / 16; ++nb2) {
         uint32_t kb[4];
         ldmatrix_x4(kb, sK + (nb2 * 16 + (lane >> 4) * 8 + (lane & 7)) * LD + ks * 16 + ((lane >> 3) & 1) * 8);
-        mma_bf16(s[2 * nb2], qf[ks], kb[0], kb[1]);
-        mma_bf16(s[2 * nb2 + 1], qf[ks], kb[2], kb[3]);
+        if (biased) {      // cached segment: FP16 operands
+          mma_f16(s[2 * nb2], qf[ks], kb[0], kb[1]);
+          mma_f16(s[2 * nb2 + 1], qf[ks], kb[2], kb[3]);
+        } else {
+          mma_bf16(s[2 * nb2], qf[ks], kb[0], kb[1]);
+          mma_bf16(s[2 * nb2 + 1], qf[ks], kb[2], kb[3]);
+        }
       }
     }
     float mx[2] = {m_run[0], m_run[1]};
@@ -262,7 +283,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
   const int n_ctiles = (p.n_cached + kBN - 1) / kBN;
   const int64_t tok_base = (int64_t)bh * p.capacity + p.cache_begin;
   if (n_ctiles > 0) {
-    load_q_frags(p.rotate ? sQr : sQ);
+    load_q_frags(sQr);
     Packed<D, BITS> pk, pv;
     // reading past n_cached stays inside `capacity` only up to the last token; clamp the index
     auto tok_of = [&](int t) { return tok_base + min((int64_t)t * kBN + key, (int64_t)p.n_cached - 1); };
@@ -270,8 +291,8 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
     load_packed<D, BITS>(pv, p.v_codes, p.v_scale, p.v_zero, tok_of(0), half, G);
     for (int t = 0; t < n_ctiles; ++t) {
       __syncthreads();
-      dequant_store<D, BITS>(pk, sK, key, half, p.group);
-      dequant_store<D, BITS>(pv, sV, key, half, p.group);
+      dequant_store<D, BITS, true>(pk, sK, key, half, p.group);
+      dequant_store<D, BITS, false>(pv, sV, key, half, p.group);
       if (half == 0) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {

@@ -27,9 +27,10 @@ def _build(B, w, chunks, tokens=None, rotate=True, signs=None, units=None, cap=N
     """GPU cache of all heads; oracle cache of `units` (or all heads); returns also the current chunk."""
     cap = cap or w.capacity
     g = B.Cache(w.batch, w.heads, w.head_dim, w.bits, w.group, cap, rotate_k=rotate, signs=signs)
-    nu = (w.batch, w.heads) if units is None else (1, len(units))
-    o = O.Cache(nu[0], nu[1], w.head_dim, w.bits, w.group, cap, rotate_k=rotate, signs=signs)
-    sel = (lambda a: a) if units is None else (lambda a: np.stack([a[b, h] for (b, h) in units])[None])
+    if units is None:
+        units = [(b, h) for b in range(w.batch) for h in range(w.heads)]
+    o = O.Cache(1, len(units), w.head_dim, w.bits, w.group, cap, rotate_k=rotate, signs=signs)
+    sel = lambda a: np.stack([a[b, h] for (b, h) in units])[None]
     n = 0
     for c in range(chunks):
         _, k, v = inputs.make_chunk(w, c, tokens=tokens)
@@ -90,7 +91,7 @@ def test_empty_cache_is_plain_attention(B):
     g = B.Cache(1, 2, 128, 2, 64, 128)
     o = O.Cache(1, 2, 128, 2, 64, 128)
     q, kc, vc = inputs.make_chunk(w, 0)
-    res = _compare(B, g, o, 0, q, kc, vc, T.sigma_of(128), lambda a: a)
+    _compare(B, g, o, 0, q, kc, vc, T.sigma_of(128), lambda a: a)
     # library attention in BF16 on the same device agrees too
     qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
     ref = torch.nn.functional.scaled_dot_product_attention(qd.float(), kd.float(), vd.float())
