@@ -10,8 +10,9 @@
 //
 // Score of a cached key (Eq. (15) / Eq. (25)):  s = sigma*q~.k^ - (sigma^2/24) sum_j step_j^2 nu_j.
 // The bias is folded into the score contraction as one extra K=16 MMA step per tile:
-// A_extra[m, j] = -(sigma/24) nu_{m,j} and B_extra[i, j] = step_{i,j}^2 (exact in BF16), so the
-// softmax warps spend no instruction on it; correction off simply skips that step.
+// A_extra[m, j] = -(sigma/24) nu_{m,j} (split into a BF16 high and low part, two columns) and
+// B_extra[i, j] = step_{i,j}^2 (exact in BF16), so the softmax warps spend no instruction on
+// it; correction off simply skips that step.
 //
 // Numerics: the rotated query and the dequantized keys are FP16 (the rotated query is not
 // representable in BF16; FP16's 11-bit significand keeps its rounding well inside the error
@@ -58,6 +59,8 @@ enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull 
 constexpr long long kTimeoutCycles = 2000000000LL;   // about a second
 constexpr long long kDrainCycles = 20000000LL;
 constexpr float kLog2e = 1.4426950408889634f;
+// registers per thread after reallocation: 128 * 72 + 256 * 168 + 128 * 96 = 64512 <= 65536
+constexpr int kRegsIssue = 72, kRegsSoftmax = 168, kRegsDequant = 96;
 constexpr float kRescaleThreshold = 8.0f;          // lazy rescale of O: only when the max grows by > 2^8
 
 struct TParams {
@@ -156,9 +159,9 @@ struct Raw {   // packed codes and metadata of one cached token (keys or values)
   uint32_t z01, z23;     // zero-points (BF16 bits) of up to 4 groups
 };
 
-template <int BITS>
+template <int BITS, int G>
 __device__ __forceinline__ void load_raw(Raw<BITS>& r, const uint8_t* codes, const uint8_t* scale, const uint16_t* zero,
-                                         int64_t tok, int G, bool valid) {
+                                         int64_t tok, bool valid) {
   if (!valid) {   // rows past the end of the cache dequantize to exact zeros
 #pragma unroll
     for (int i = 0; i < Raw<BITS>::kWords; ++i) r.w[i] = 0;
@@ -171,9 +174,9 @@ __device__ __forceinline__ void load_raw(Raw<BITS>& r, const uint8_t* codes, con
     const uint4 v = __ldg(cw + i);
     r.w[4 * i] = v.x; r.w[4 * i + 1] = v.y; r.w[4 * i + 2] = v.z; r.w[4 * i + 3] = v.w;
   }
-  if (G == 1) {
+  if constexpr (G == 1) {
     r.sbytes = __ldg(scale + tok); r.z01 = __ldg(zero + tok); r.z23 = 0;
-  } else if (G == 2) {
+  } else if constexpr (G == 2) {
     r.sbytes = __ldg(reinterpret_cast<const uint16_t*>(scale + tok * 2));
     r.z01 = __ldg(reinterpret_cast<const uint32_t*>(zero + tok * 2)); r.z23 = 0;
   } else {
@@ -195,8 +198,9 @@ __device__ __forceinline__ float raw_zero(const Raw<BITS>& r, int j) {
 // with OFF = 4 (2-bit) or 16 (4-bit) coming for free from the exponent bits OR-ed over the code.
 // Pairs are (i, i + 8) of each 16-code word (2-bit) or (i, i + 4) of each 8-code word (4-bit): the
 // contraction dimension is stored permuted, and the rotated query is stored with the same permutation.
-template <int BITS>
-__device__ __forceinline__ void dequant_keys(const Raw<BITS>& r, uint8_t* tile, int key, int group) {
+template <int BITS, int GROUP>
+__device__ __forceinline__ void dequant_keys(const Raw<BITS>& r, uint8_t* tile, int key) {
+  constexpr int group = GROUP;
   constexpr float kOff = (BITS == 2) ? 4.f : 16.f;
   uint32_t step2[4], c2[4];
 #pragma unroll
@@ -239,8 +243,9 @@ __device__ __forceinline__ void dequant_keys(const Raw<BITS>& r, uint8_t* tile, 
 // Values: same reconstruction as BF16, channels in natural order (the output dimension cannot be permuted
 // because current-chunk values arrive unpermuted).  2-bit: one FMA per pair; 4-bit: exact subtract then
 // multiply (the 16 + zero offset times the step is not always representable in BF16).
-template <int BITS>
-__device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile, int key, int group) {
+template <int BITS, int GROUP>
+__device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile, int key) {
+  constexpr int group = GROUP;
   uint32_t step2[4], c2[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
@@ -287,7 +292,7 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
   }
 }
 
-template <int BITS>
+template <int BITS, int GROUP>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const TParams p) {
@@ -303,7 +308,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int n_rt = (p.n_cur + kBlockN - 1) / kBlockN;
   const int n_ct = (p.n_cached + kBlockN - 1) / kBlockN;
   const int T = n_rt + n_ct;
-  const int G = kD / p.group;
+  constexpr int G = kD / GROUP;
 
   if (tid == 0) {
     misc[1] = 0;
@@ -337,6 +342,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
   // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_q aliases the first 64 columns of S_q.
 
+  if (warp < 4) {
+    setmaxnreg_dec<kRegsIssue>();
   if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
@@ -449,8 +456,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       tc_commit(cx.bar(kDrain));
       cx.drain(kDrain, 0);
     }
-  } else if (warp >= 4 && warp < 12) {
+  }
+  } else if (warp < 12) {
     // ================= softmax groups =================
+    setmaxnreg_inc<kRegsSoftmax>();
     const int qt = (warp - 4) >> 2;
     const int wq = warp & 3;
     const int r_in_tile = wq * 32 + lane;
@@ -467,54 +476,53 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       ok = __all_sync(0xFFFFFFFFu, cx.wait(kSFull + qt, t & 1, 301));
       if (!ok) break;
       tc_fence_after();
-      uint32_t r[32];
-      float mx = -INFINITY;
+      uint32_t sr[128];                          // this row's 128 scores, then its 64 packed probabilities
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(s_addr + 32 * c, r);
-        tmem_wait_ld();
+      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + 32 * c, sr + 32 * c);
+      tmem_wait_ld();
+      if (n_valid < kBlockN) {                   // ragged last tile of a segment
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float v = (32 * c + i < n_valid) ? __uint_as_float(r[i]) : -INFINITY;
-          mx = fmaxf(mx, v);
-        }
+        for (int i = 0; i < 128; ++i)
+          if (i >= n_valid) sr[i] = 0xFF800000u;  // -inf
       }
-      const float m_new = fmaxf(m, mx * c_row);
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i += 4) {
+        mx0 = max3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+        mx1 = max3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+      }
+      const float m_new = fmaxf(m, fmaxf(mx0, mx1) * c_row);
       if (__any_sync(0xFFFFFFFFu, m_new - m > kRescaleThreshold)) {
         if (t > 0) {
           ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (t - 1) & 1, 302));
           if (!ok) break;
           tc_fence_after();
           const float f = ex2(m - m_new);
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            tmem_ld32(o_addr + 32 * c, r);
+#pragma unroll 1
+          for (int c = 0; c < 8; ++c) {
+            uint32_t r[16];
+            tmem_ld16(o_addr + 16 * c, r);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-            tmem_st32(o_addr + 32 * c, r);
+            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+            tmem_st16(o_addr + 16 * c, r);
           }
           l_cur *= f; l_cac *= f;
         }
         m = m_new;
       }
-      float sum = 0.f;
+      const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m, -m);
+      float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(s_addr + 32 * c, r);
-        tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float x0 = (32 * c + i < n_valid) ? fmaf(__uint_as_float(r[i]), c_row, -m) : -INFINITY;
-          const float x1 = (32 * c + i + 1 < n_valid) ? fmaf(__uint_as_float(r[i + 1]), c_row, -m) : -INFINITY;
-          const float p0 = ex2(x0), p1 = ex2(x1);
-          sum += p0 + p1;
-          pk[i >> 1] = pack_bf16x2(p0, p1);
-        }
-        tmem_st16(s_addr + 16 * c, pk);
+      for (int i = 0; i < 128; i += 2) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), c2, nm2);
+        const float p0 = ex2(x.x), p1 = ex2(x.y);
+        sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
+        sr[i >> 1] = cvt_bf16x2(p0, p1);
       }
-      if (cached) l_cac += sum; else l_cur += sum;
+      tmem_st32(s_addr, sr);
+      tmem_st32(s_addr + 32, sr + 32);
+      if (cached) l_cac += sum2.x + sum2.y; else l_cur += sum2.x + sum2.y;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(cx.bar(kPFull + qt));
@@ -549,15 +557,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
     }
     tc_fence_before();
-  } else if (warp >= 12) {
+  } else {
     // ================= dequant + query rotation =================
+    setmaxnreg_dec<kRegsDequant>();
     const int dt = tid - 12 * 32;          // 0..127: the key of the tile this thread expands
     const int64_t tok0 = (int64_t)bh * p.capacity + p.cache_begin;
     Raw<BITS> rk, rv;
     if (n_ct > 0) {
       const bool valid = dt < p.n_cached;
-      load_raw<BITS>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + dt, G, valid);
-      load_raw<BITS>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + dt, G, valid);
+      load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + dt, valid);
+      load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + dt, valid);
     }
     bool ok = true;
     for (int t = 0; t < T; ++t) {
@@ -567,16 +576,17 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       ok = __all_sync(0xFFFFFFFFu, cx.wait(kKEmpty + s, ph ^ 1, 401));
       if (!ok) break;
       if (ct >= 0) {
-        dequant_keys<BITS>(rk, smem + kOffK + s * kTileBytes, dt, p.group);
+        dequant_keys<BITS, GROUP>(rk, smem + kOffK + s * kTileBytes, dt);
         if (p.correction) {   // B_extra row: step_j^2, exact in BF16
           const float d0 = raw_step<BITS>(rk, 0), d1 = raw_step<BITS>(rk, 1), d2 = raw_step<BITS>(rk, 2), d3 = raw_step<BITS>(rk, 3);
-          *reinterpret_cast<uint2*>(smem + kOffBx + s * kXBytes + xtile_offset(dt, 0)) =
-              make_uint2(pack_bf16x2(d0 * d0, G > 1 ? d1 * d1 : 0.f), pack_bf16x2(G > 2 ? d2 * d2 : 0.f, G > 3 ? d3 * d3 : 0.f));
+          const uint32_t b01 = pack_bf16x2(d0 * d0, G > 1 ? d1 * d1 : 0.f), b23 = pack_bf16x2(G > 2 ? d2 * d2 : 0.f, G > 3 ? d3 * d3 : 0.f);
+          // columns 0..3 meet the high parts of A_extra, columns 4..7 the low parts
+          *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(dt, 0)) = make_uint4(b01, b23, b01, b23);
         }
         fence_proxy_async_smem();
         if (ct + 1 < n_ct) {
           const int k1 = (ct + 1) * kBlockN + dt;
-          load_raw<BITS>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k1, G, k1 < p.n_cached);
+          load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k1, k1 < p.n_cached);
         }
       }
       mbar_arrive(cx.bar(kKFull + s));
@@ -585,7 +595,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, 0, 402) && cx.wait(kQCurDone, 0, 403));
         if (!ok) break;
         const int l16 = lane & 15, rsub = lane >> 4;
-        const int lanes_per_group = p.group / 8;
+        constexpr int lanes_per_group = GROUP / 8;
         float sgn[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) sgn[e] = (p.rotate && p.signs) ? (float)p.signs[l16 * 8 + e] : 1.0f;
@@ -623,8 +633,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int off = 1; off < lanes_per_group; off *= 2) nu += __shfl_xor_sync(0xFFFFFFFFu, nu, off);
           if ((l16 % lanes_per_group) == 0) {
             const int j = l16 / lanes_per_group;
-            *reinterpret_cast<uint16_t*>(smem + kOffAx + qt * kXBytes + xtile_offset(rr, 0) + 2 * j) =
-                (uint16_t)f32_to_bf16_bits(p.ax_coef * nu);
+            // -(sigma/24) nu as a BF16 high part plus a BF16 low part (columns j and 4 + j)
+            const float a = p.ax_coef * nu;
+            const uint32_t hi = f32_to_bf16_bits(a);
+            uint8_t* ax = smem + kOffAx + qt * kXBytes + xtile_offset(rr, 0);
+            *reinterpret_cast<uint16_t*>(ax + 2 * j) = (uint16_t)hi;
+            *reinterpret_cast<uint16_t*>(ax + 8 + 2 * j) = (uint16_t)f32_to_bf16_bits(a - bf16_bits_to_f32(hi));
           }
           float y[8];
           if constexpr (BITS == 2) {
@@ -653,11 +667,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       ok = __all_sync(0xFFFFFFFFu, cx.wait(kVEmpty + s, ph ^ 1, 404));
       if (!ok) break;
       if (ct >= 0) {
-        dequant_values<BITS>(rv, smem + kOffV + s * kTileBytes, dt, p.group);
+        dequant_values<BITS, GROUP>(rv, smem + kOffV + s * kTileBytes, dt);
         fence_proxy_async_smem();
         if (ct + 1 < n_ct) {
           const int k1 = (ct + 1) * kBlockN + dt;
-          load_raw<BITS>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k1, G, k1 < p.n_cached);
+          load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k1, k1 < p.n_cached);
         }
       }
       mbar_arrive(cx.bar(kVFull + s));
@@ -709,14 +723,14 @@ int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, kvq_strides s
   return KVQ_OK;
 }
 
-template <int BITS>
+template <int BITS, int GROUP>
 int launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TParams& p, dim3 grid, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
-    KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_tcgen05_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_tcgen05_kernel<BITS, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured = true;
   }
-  attn_tcgen05_kernel<BITS><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
+  attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
   KVQ_CUDA_TRY(cudaGetLastError());
   return KVQ_OK;
 }
@@ -752,7 +766,14 @@ int launch_attn_tcgen05(const AttnArgs& a) {
   p.ax_coef = -a.softmax_scale / 24.0f;
   p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
   dim3 grid((unsigned)((a.m_tokens + 2 * kBlockM - 1) / (2 * kBlockM)), (unsigned)((int64_t)d->batch * d->heads));
-  return d->bits == 2 ? launch<2>(mq, mk, mv, p, grid, a.stream) : launch<4>(mq, mk, mv, p, grid, a.stream);
+  if (d->bits == 2) {
+    if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
+    if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);
+    return launch<2, 128>(mq, mk, mv, p, grid, a.stream);
+  }
+  if (d->group == 32) return launch<4, 32>(mq, mk, mv, p, grid, a.stream);
+  if (d->group == 64) return launch<4, 64>(mq, mk, mv, p, grid, a.stream);
+  return launch<4, 128>(mq, mk, mv, p, grid, a.stream);
 }
 
 }  // namespace kvq

@@ -19,8 +19,12 @@ def B():
     return binding
 
 
-def kernels(B):
-    return [("auto", B.KVQ_KERNEL_AUTO), ("mma_sync", B.KVQ_KERNEL_MMA_SYNC)]
+def kernels(B, head_dim=128):
+    """Every kernel that covers the shape: the warp-level one always, the tcgen05 one for head_dim 128."""
+    ks = [("mma_sync", B.KVQ_KERNEL_MMA_SYNC)]
+    if head_dim == 128:
+        ks.append(("tcgen05", B.KVQ_KERNEL_TCGEN05))
+    return ks
 
 
 def _build(B, w, chunks, tokens=None, rotate=True, signs=None, units=None, cap=None):
@@ -44,7 +48,7 @@ def _compare(B, g, o, n_cache, q, kc, vc, sigma, sel, rows=None, flags_list=None
     res = {}
     for corr in (True, False):
         want = O.attn_corrected(o, begin, n_cache, sel(q), sel(kc), sel(vc), sigma, correction=corr, rows=rows)
-        for kname, kflag in (flags_list or kernels(B)):
+        for kname, kflag in (flags_list or kernels(B, q.shape[-1])):
             flags = (B.KVQ_CORRECTION_ON if corr else B.KVQ_CORRECTION_OFF) | kflag
             lse = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
             mass = torch.zeros_like(lse)
@@ -106,7 +110,7 @@ def test_zero_steps_make_correction_a_noop(B):
     o.k_scale[:] = 0
     q, kc, vc = inputs.make_chunk(w, 3)
     qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
-    for _, kflag in kernels(B):
+    for _, kflag in kernels(B, 128):
         on = B.kvq_attn_corrected(g, qd, kd, vd, T.sigma_of(128), B.KVQ_CORRECTION_ON | kflag)
         off = B.kvq_attn_corrected(g, qd, kd, vd, T.sigma_of(128), B.KVQ_CORRECTION_OFF | kflag)
         assert torch.equal(on, off) and torch.isfinite(on.float()).all()
@@ -128,6 +132,20 @@ def test_rotation_off_window_scale_and_strides(B):
     B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON, cache_begin=48, cache_len=150, out=out)
     want = O.attn_corrected(o, 48, 150, q, kc, vc, sigma, correction=True)["out"]
     T.assert_attn_close(T.from_dev_bf16(out), want, "strided")
+
+
+def test_auto_dispatch_and_forced_kernel_errors(B):
+    # head_dim 128 -> tcgen05 kernel, head_dim 64 -> warp-level kernel; forcing tcgen05 on 64 is refused
+    for d in (64, 128):
+        w = inputs.Workload("auto", 310 + d, 1, 2, d, 140, 0, 2, 64, 0)
+        g, o, n, sel = _build(B, w, 2, tokens=90, cap=256)
+        q, kc, vc = inputs.make_chunk(w, 3)
+        _compare(B, g, o, n, q, kc, vc, T.sigma_of(d), sel, flags_list=[("auto", B.KVQ_KERNEL_AUTO)])
+        if d == 64:
+            with pytest.raises(B.KvqError) as e:
+                B.kvq_attn_corrected(g, T.to_dev(q), T.to_dev(kc), T.to_dev(vc), 0.125,
+                                     B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05)
+            assert e.value.status == B.KVQ_ERR_UNSUPPORTED
 
 
 def test_correction_lowers_cached_mass_and_mass_is_consistent(B):
