@@ -20,7 +20,6 @@ import math
 import os
 import subprocess
 import sys
-import threading
 import time
 
 import numpy as np
@@ -53,21 +52,18 @@ class ClockSampler:
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
+        import tempfile
         self.index, self.proc, self.lines = index, None, []
+        self.path = os.path.join(tempfile.gettempdir(), f"kvq_clocks_{os.getpid()}_{index}.csv")
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-i", str(self.index),
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.t = threading.Thread(target=self._read, daemon=True)
-            self.t.start()
+                 "-lms", "50", "-f", self.path], stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+            time.sleep(0.3)
         except OSError:
             self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
 
     def stop(self):
         if not self.proc:
@@ -77,6 +73,12 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        try:
+            with open(self.path) as f:
+                self.lines = [ln.strip() for ln in f]
+            os.remove(self.path)
+        except OSError:
+            self.lines = []
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for ln in self.lines:
@@ -141,10 +143,14 @@ def main():
     ap.add_argument("--impl", default="kvq", choices=["kvq", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="only warm-up and timed steps (no correction-off, end-to-end or CPU legs): the command to run under ncu")
     args = ap.parse_args()
 
     from paper_2605_26266_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
+    if args.profile:
+        args.no_e2e = args.no_cpu_baseline = True
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -238,7 +244,7 @@ def main():
 
     # correction off, same kernel: cost of the correction
     recs_off = []
-    for i in range(max(3, min(args.steps, 20)) + 3):
+    for i in range(0 if args.profile else max(3, min(args.steps, 20)) + 3):
         flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -247,7 +253,7 @@ def main():
         if i >= 3:
             recs_off.append((e0, e1))
     torch.cuda.synchronize()
-    attn_off_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in recs_off]))
+    attn_off_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in recs_off])) if recs_off else float("nan")
 
     # ---- end to end through the public call with HOST buffers ----
     e2e = None
