@@ -1,7 +1,7 @@
 // Corrected chunk attention for sm_100a: TMA + tcgen05.mma with TMEM accumulators.
 //
-// One CTA owns 256 query rows of one (batch, head) — two 128-row tiles that ping-pong on the
-// tensor pipe — and walks all keys in tiles of 128: first the current chunk's BF16 keys and
+// A CTA works on 256 query rows of one (batch, head) at a time — two 128-row tiles that ping-pong on the
+// tensor pipe — and walks keys in tiles of 128: first the current chunk's BF16 keys and
 // values (TMA straight into the 128-byte-swizzled operand layout, unrotated query, no bias),
 // then the cached keys and values, which four "dequant" warps expand from the packed
 // 2-/4-bit codes into the same operand layout in shared memory (never to HBM).  Between the
@@ -21,11 +21,20 @@
 // columns and consumed from there by the PV MMA.  Rotated queries are clamped to the FP16
 // range; dequantized keys must lie inside it.
 //
-// Roles (512 threads): warp 0 lane 0 issues TMA, warp 1 lane 0 issues all MMAs, warps 4-7 and
-// 8-11 are the softmax groups of query tile 0 and 1 (one thread per row = one TMEM lane),
-// warps 12-15 dequantize and rotate.  Every wait on an mbarrier is bounded: on expiry the CTA
-// records a diagnostic in the caller's status word, all roles leave their loops, in-flight
-// work is drained with a bounded wait, TMEM is freed and the kernel returns.
+// Roles (512 threads): warp 0 lane 0 issues TMA; warp 1 runs the MMA schedule converged and one elected
+// lane issues every tcgen05.mma; warps 4-11 are the softmax warps: warp 4+q and warp 8+q share TMEM lanes
+// 32q..32q+31 (one query row per lane) and take columns [0,64) and [64,128) of each score tile, exchanging
+// their partial row maxima through shared memory, for both query tiles in turn; warps 12-15 dequantize
+// and rotate.  Registers are re-split between the roles with setmaxnreg.
+//
+// Work is cut into units (batch*head, 256-row query block) of `tiles` key tiles each.  When units are
+// plentiful a CTA computes one whole unit; otherwise the unit x tile steps are divided evenly over one CTA
+// per SM, a CTA walks its range segment by segment, split units leave unnormalised partial results
+// (O, running max, row sums) in the caller's workspace and a small second kernel merges them.
+//
+// Every wait on an mbarrier is bounded: on expiry the CTA records a diagnostic in the caller's status
+// word, all roles leave their loops, in-flight work is drained with a bounded wait, TMEM is freed and the
+// kernel returns.
 #include <cuda_fp16.h>
 
 #include "kvq_common.cuh"
@@ -49,18 +58,22 @@ constexpr int kOffV = kOffK + 2 * kTileBytes;      // 2 stages
 constexpr int kOffAx = kOffV + 2 * kTileBytes;     // 2 query tiles
 constexpr int kOffBx = kOffAx + 2 * kXBytes;       // 2 stages
 constexpr int kOffBar = kOffBx + 2 * kXBytes;
-constexpr int kNumBars = 20;
-constexpr int kOffMisc = kOffBar + kNumBars * 8;
+constexpr int kNumBars = 30;
+constexpr int kOffXmax = kOffBar + 256;            // float [2 column halves][256 rows]: row-max exchange
+constexpr int kOffXl = kOffXmax + 2 * 256 * 4;     // float [2][256][2]: row-sum exchange (current, cached)
+constexpr int kOffMisc = kOffXl + 2 * 256 * 2 * 4;
 constexpr int kSmemBytes = kOffMisc + 64 + 1024;   // + slack to align the base to 1024
 
 enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull = 9, kPFull = 11,
-           kODone = 13, kQCurDone = 15, kQRotFull = 16, kDrain = 17 };
+           kODone = 13, kQCurDone = 15, kQRotFull = 16, kDrain = 17, kQEmpty = 18, kOFree = 19,
+           kPair = 21 /* 8: [query tile][lane quarter], the two warps that share 32 rows */ };
 
 constexpr long long kTimeoutCycles = 2000000000LL;   // about a second
 constexpr long long kDrainCycles = 20000000LL;
 constexpr float kLog2e = 1.4426950408889634f;
 // registers per thread after reallocation: 128 * 72 + 256 * 168 + 128 * 96 = 64512 <= 65536
 constexpr int kRegsIssue = 72, kRegsSoftmax = 168, kRegsDequant = 96;
+constexpr uint32_t kFmaPipePairs = 0x00000000u;      // which of a thread's 32 score pairs use exp2_fma_pipe
 constexpr float kRescaleThreshold = 8.0f;          // lazy rescale of O: only when the max grows by > 2^8
 
 struct TParams {
@@ -75,6 +88,33 @@ struct TParams {
   float ax_coef;           // -sigma / 24
   float* lse; float* cached_mass;
   int32_t* status;
+  // persistent schedule: units = (batch*head, 256-row query block); every unit has `tiles` key tiles;
+  // the n_units * tiles tile steps are cut into gridDim.x equal contiguous ranges
+  int q_blocks, n_units, tiles;
+  float* partial;          // workspace: 2 slots per CTA, see kSlotFloats
+};
+
+// One partial result: unnormalised O [256][128] FP32, then m[256], l_cur[256], l_cached[256]
+constexpr int kSlotFloats = 256 * kD + 3 * 256;
+
+// A contiguous run of key tiles [tb, te) of one unit.
+struct Segment { int unit, tb, te; };
+struct Schedule {
+  int g, g_end, tiles;     // n_units * tiles < 2^31 (checked on the host)
+  __device__ __forceinline__ Schedule(int cta, int n_ctas, int n_units, int tiles_) : tiles(tiles_) {
+    const long long W = (long long)n_units * tiles_;
+    g = (int)(W * cta / n_ctas);
+    g_end = (int)(W * (cta + 1) / n_ctas);
+  }
+  __device__ __forceinline__ bool next(Segment& sg) {
+    if (g >= g_end) return false;
+    sg.unit = g / tiles;
+    sg.tb = g - sg.unit * tiles;
+    const int n = min(tiles - sg.tb, g_end - g);
+    sg.te = sg.tb + n;
+    g += n;
+    return true;
+  }
 };
 
 struct Ctx {
@@ -117,6 +157,21 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// 2^x for a pair on the FMA pipe instead of the MUFU: round-to-nearest split x = n + r, |r| <= 1/2, a cubic
+// for 2^r (relative error 7.5e-5, well below BF16 resolution of the probabilities) and an integer add of
+// n into the exponent field.  Inputs are clamped at -126 (results that small are zero for our purposes).
+__device__ __forceinline__ float2 exp2_fma_pipe(float2 x) {
+  x.x = fmaxf(x.x, -126.f); x.y = fmaxf(x.y, -126.f);
+  const float kMagic = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+  const float2 r = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+  float2 q = __ffma2_rn(make_float2(0.05517164617776871f, 0.05517164617776871f), r, make_float2(0.2426111251115799f, 0.2426111251115799f));
+  q = __ffma2_rn(q, r, make_float2(0.6932609677314758f, 0.6932609677314758f));
+  q = __ffma2_rn(q, r, make_float2(0.9999280571937561f, 0.9999280571937561f));
+  return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23)),
+                     __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23)));
 }
 __device__ __forceinline__ uint32_t hfma2_f16(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t d;
@@ -292,6 +347,80 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
   }
 }
 
+// Rotates the CTA's 256-row query tile in place (four warps; 16 lanes per row, 8 channels per lane):
+// q~ = (1/sqrt d) H (signs . q) in FP32, written back as FP16 with the contraction dimension permuted the
+// way the dequantized keys are laid out, and -(sigma/24) nu_{m,j} written to the bias operand tile.
+template <int BITS, int GROUP>
+__device__ __forceinline__ void rotate_query(uint8_t* smem, const TParams& p, int warp, int lane) {
+    const int l16 = lane & 15, rsub = lane >> 4;
+    constexpr int lanes_per_group = GROUP / 8;
+    float sgn[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sgn[e] = (p.rotate && p.signs) ? (float)p.signs[l16 * 8 + e] : 1.0f;
+    for (int pass = 0; pass < 32; ++pass) {
+      const int qrow = pass * 8 + (warp - 12) * 2 + rsub;     // 0..255
+      const int qt = qrow >> 7, rr = qrow & 127;
+      uint8_t* qtile = smem + kOffQ + qt * kTileBytes;
+      const uint4 raw = *reinterpret_cast<const uint4*>(qtile + sw128_offset(rr, l16));
+      float x[8];
+      x[0] = bf16_bits_to_f32(raw.x & 0xFFFFu); x[1] = bf16_bits_to_f32(raw.x >> 16);
+      x[2] = bf16_bits_to_f32(raw.y & 0xFFFFu); x[3] = bf16_bits_to_f32(raw.y >> 16);
+      x[4] = bf16_bits_to_f32(raw.z & 0xFFFFu); x[5] = bf16_bits_to_f32(raw.z >> 16);
+      x[6] = bf16_bits_to_f32(raw.w & 0xFFFFu); x[7] = bf16_bits_to_f32(raw.w >> 16);
+      if (p.rotate) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] *= sgn[e];
+#pragma unroll
+        for (int hh = 1; hh < 8; hh *= 2)
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if ((i & hh) == 0) { const float a = x[i], c = x[i + hh]; x[i] = a + c; x[i + hh] = a - c; }
+#pragma unroll
+        for (int lm = 1; lm < 16; lm *= 2)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
+            x[e] = (l16 & lm) ? (o - x[e]) : (x[e] + o);
+          }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] *= 0.08838834764831845f;
+      }
+      float nu = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) nu += x[e] * x[e];
+      for (int off = 1; off < lanes_per_group; off *= 2) nu += __shfl_xor_sync(0xFFFFFFFFu, nu, off);
+      if ((l16 % lanes_per_group) == 0) {
+        const int j = l16 / lanes_per_group;
+        // -(sigma/24) nu as a BF16 high part plus a BF16 low part (columns j and 4 + j)
+        const float a = p.ax_coef * nu;
+        const uint32_t hi = f32_to_bf16_bits(a);
+        uint8_t* ax = smem + kOffAx + qt * kXBytes + xtile_offset(rr, 0);
+        *reinterpret_cast<uint16_t*>(ax + 2 * j) = (uint16_t)hi;
+        *reinterpret_cast<uint16_t*>(ax + 8 + 2 * j) = (uint16_t)f32_to_bf16_bits(a - bf16_bits_to_f32(hi));
+      }
+      float y[8];
+      if constexpr (BITS == 2) {
+        // physical column 16w + 2i + hsel <- channel 16w + i + 8*hsel: even lanes own the low half
+        // of a 16-channel word, odd lanes the high half; swap four values with the neighbour
+        const bool odd = l16 & 1;
+        float rcv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) rcv[i] = __shfl_xor_sync(0xFFFFFFFFu, odd ? x[i] : x[4 + i], 1);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          y[2 * i] = odd ? rcv[i] : x[i];
+          y[2 * i + 1] = odd ? x[4 + i] : rcv[i];
+        }
+      } else {
+        // physical column 8w + 2i + hsel <- channel 8w + i + 4*hsel
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { y[2 * i] = x[i]; y[2 * i + 1] = x[4 + i]; }
+      }
+      *reinterpret_cast<uint4*>(qtile + sw128_offset(rr, l16)) =
+          make_uint4(pack_f16x2_sat(y[0], y[1]), pack_f16x2_sat(y[2], y[3]), pack_f16x2_sat(y[4], y[5]), pack_f16x2_sat(y[6], y[7]));
+    }
+}
+
 template <int BITS, int GROUP>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -303,8 +432,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   Ctx cx{sbase + kOffBar, misc + 1, p.status};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int bh = blockIdx.y, b = bh / p.heads, h = bh - b * p.heads;
-  const int row0 = blockIdx.x * (2 * kBlockM);
   const int n_rt = (p.n_cur + kBlockN - 1) / kBlockN;
   const int n_ct = (p.n_cached + kBlockN - 1) / kBlockN;
   const int T = n_rt + n_ct;
@@ -319,12 +446,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_init(cx.bar(kKEmpty + s), 1);
       mbar_init(cx.bar(kVEmpty + s), 1);
       mbar_init(cx.bar(kSFull + s), 1);
-      mbar_init(cx.bar(kPFull + s), 128);
+      mbar_init(cx.bar(kPFull + s), 256);
       mbar_init(cx.bar(kODone + s), 1);
     }
     mbar_init(cx.bar(kQCurDone), 1);
     mbar_init(cx.bar(kQRotFull), 128);
     mbar_init(cx.bar(kDrain), 1);
+    mbar_init(cx.bar(kQEmpty), 1);
+    mbar_init(cx.bar(kOFree + 0), 256);
+    mbar_init(cx.bar(kOFree + 1), 256);
+    for (int i = 0; i < 8; ++i) mbar_init(cx.bar(kPair + i), 64);
     fence_barrier_init();
     prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
   }
@@ -347,334 +478,380 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
-      mbar_arrive_expect_tx(cx.bar(kQFull), 2 * kTileBytes);
-      for (int qt = 0; qt < 2; ++qt)
-        for (int kb = 0; kb < 2; ++kb)
-          tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, &tm_q, cx.bar(kQFull), kb * 64, row0 + qt * kBlockM, h, b);
-      int issued = 0;
-      for (int t = 0; t < T; ++t) {
-        const int s = t & 1;
-        const uint32_t ph = (t >> 1) & 1;
-        if (!cx.wait(kKEmpty + s, ph ^ 1, 101)) break;
-        if (t < n_rt) {
-          mbar_arrive_expect_tx(cx.bar(kKFull + s), kTileBytes);
+      Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+      Segment sg;
+      int it = 0, nseg = 0, issued_it = -1;
+      bool ok = true;
+      while (ok && sch.next(sg)) {
+        const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
+        const int row0 = (sg.unit - bh * p.q_blocks) * (2 * kBlockM);
+        // the query buffer is free once every score MMA of the previous segment has retired
+        if (!(ok = cx.wait(kQEmpty, (nseg & 1) ^ 1, 100))) break;
+        mbar_arrive_expect_tx(cx.bar(kQFull), 2 * kTileBytes);
+        for (int qt = 0; qt < 2; ++qt)
           for (int kb = 0; kb < 2; ++kb)
-            tma_load_4d(sbase + kOffK + s * kTileBytes + kb * kHalfTile, &tm_k, cx.bar(kKFull + s), kb * 64, t * kBlockN, h, b);
-        } else {
-          mbar_arrive(cx.bar(kKFull + s));
+            tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, &tm_q, cx.bar(kQFull), kb * 64, row0 + qt * kBlockM, h, b);
+        for (int t = sg.tb; t < sg.te; ++t, ++it) {
+          const int s = it & 1;
+          const uint32_t ph = (it >> 1) & 1;
+          if (!(ok = cx.wait(kKEmpty + s, ph ^ 1, 101))) break;
+          if (t < n_rt) {
+            mbar_arrive_expect_tx(cx.bar(kKFull + s), kTileBytes);
+            for (int kb = 0; kb < 2; ++kb)
+              tma_load_4d(sbase + kOffK + s * kTileBytes + kb * kHalfTile, &tm_k, cx.bar(kKFull + s), kb * 64, t * kBlockN, h, b);
+          } else {
+            mbar_arrive(cx.bar(kKFull + s));
+          }
+          if (!(ok = cx.wait(kVEmpty + s, ph ^ 1, 102))) break;
+          if (t < n_rt) {
+            mbar_arrive_expect_tx(cx.bar(kVFull + s), kTileBytes);
+            for (int kb = 0; kb < 2; ++kb)
+              tma_load_4d(sbase + kOffV + s * kTileBytes + kb * kHalfTile, &tm_v, cx.bar(kVFull + s), kb * 64, t * kBlockN, h, b);
+            issued_it = it;
+          } else {
+            mbar_arrive(cx.bar(kVFull + s));
+          }
         }
-        if (!cx.wait(kVEmpty + s, ph ^ 1, 102)) break;
-        if (t < n_rt) {
-          mbar_arrive_expect_tx(cx.bar(kVFull + s), kTileBytes);
-          for (int kb = 0; kb < 2; ++kb)
-            tma_load_4d(sbase + kOffV + s * kTileBytes + kb * kHalfTile, &tm_v, cx.bar(kVFull + s), kb * 64, t * kBlockN, h, b);
-          issued = t + 1;
-        } else {
-          mbar_arrive(cx.bar(kVFull + s));
-        }
+        ++nseg;
       }
       if (*cx.abort) {   // drain: give loads already in flight a bounded time to land before the CTA exits
-        cx.drain(kQFull, 0);
-        for (int t = max(0, issued - 2); t < issued; ++t) {
-          cx.drain(kKFull + (t & 1), (t >> 1) & 1);
-          cx.drain(kVFull + (t & 1), (t >> 1) & 1);
+        if (nseg > 0) cx.drain(kQFull, (nseg - 1) & 1);
+        if (issued_it >= 0) {
+          cx.drain(kKFull + (issued_it & 1), (issued_it >> 1) & 1);
+          cx.drain(kVFull + (issued_it & 1), (issued_it >> 1) & 1);
         }
       }
     }
   } else if (warp == 1) {
     // ================= MMA issuer =================
-    if (lane == 0) {
+    // The whole warp runs this code converged (operands stay warp-uniform); one elected lane issues.
+    {
       const uint32_t idesc_bf16 = make_idesc_bf16(128, 128, 0, 0);
       const uint32_t idesc_f16 = idesc_bf16 & ~((7u << 7) | (7u << 10));     // A, B format 0 = FP16
       const uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);              // B (values) is MN-major
-      auto issue_qk = [&](int qt, int t) {
-        const int s = t & 1;
-        const bool cached = t >= n_rt;
+      // Descriptors are built once; stepping along K only adds a constant to the 14-bit address field
+      // (all operand tiles live below 256 KiB of shared memory, so the field cannot overflow).
+      const uint64_t dq0 = make_smem_desc(sbase + kOffQ, 16, 1024, kLayoutSw128);
+      const uint64_t dk0 = make_smem_desc(sbase + kOffK, 16, 1024, kLayoutSw128);
+      const uint64_t dv0 = make_smem_desc(sbase + kOffV, kHalfTile, 1024, kLayoutSw128);
+      const uint64_t dax0 = make_smem_desc(sbase + kOffAx, 128, 256, kLayoutNone);
+      const uint64_t dbx0 = make_smem_desc(sbase + kOffBx, 128, 256, kLayoutNone);
+      auto commit1 = [&](uint32_t bar) { if (elect_one()) tc_commit(bar); __syncwarp(); };
+      auto issue_qk = [&](int qt, int s, bool cached) {
+        if (elect_one()) {
         const uint32_t idesc = cached ? idesc_f16 : idesc_bf16;
-        const uint32_t qa = sbase + kOffQ + qt * kTileBytes, ka = sbase + kOffK + s * kTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t off = (ks >> 2) * kHalfTile + (ks & 3) * 32;
-          mma_ss(tmem + qt * 128, make_smem_desc(qa + off, 16, 1024, kLayoutSw128),
-                 make_smem_desc(ka + off, 16, 1024, kLayoutSw128), idesc, ks > 0);
-        }
+        const uint64_t qd = dq0 + (uint64_t)(qt * (kTileBytes >> 4)), kd = dk0 + (uint64_t)(s * (kTileBytes >> 4));
+        const uint32_t d_tmem = tmem + qt * 128;
+        constexpr int kBlk = kHalfTile >> 4;
+        mma_ss_off<0>(d_tmem, qd, kd, idesc, 0);
+        mma_ss_off<2>(d_tmem, qd, kd, idesc, 1);
+        mma_ss_off<4>(d_tmem, qd, kd, idesc, 1);
+        mma_ss_off<6>(d_tmem, qd, kd, idesc, 1);
+        mma_ss_off<kBlk>(d_tmem, qd, kd, idesc, 1);
+        mma_ss_off<kBlk + 2>(d_tmem, qd, kd, idesc, 1);
+        mma_ss_off<kBlk + 4>(d_tmem, qd, kd, idesc, 1);
+        mma_ss_off<kBlk + 6>(d_tmem, qd, kd, idesc, 1);
         if (cached && p.correction)
-          mma_ss(tmem + qt * 128, make_smem_desc(sbase + kOffAx + qt * kXBytes, 128, 256, kLayoutNone),
-                 make_smem_desc(sbase + kOffBx + s * kXBytes, 128, 256, kLayoutNone), idesc_bf16, 1);
+          mma_ss(d_tmem, dax0 + (uint64_t)(qt * (kXBytes >> 4)), dbx0 + (uint64_t)(s * (kXBytes >> 4)), idesc_bf16, 1);
         tc_commit(cx.bar(kSFull + qt));
+        }
+        __syncwarp();
       };
-      auto issue_pv = [&](int qt, int t) {
-        const int s = t & 1;
-        const uint32_t va = sbase + kOffV + s * kTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          mma_ts(tmem + 256 + qt * 128, tmem + qt * 128 + ks * 8,
-                 make_smem_desc(va + ks * 2048, kHalfTile, 1024, kLayoutSw128), idesc_pv, (t > 0 || ks > 0));
+      auto issue_pv = [&](int qt, int s, bool accumulate) {
+        if (elect_one()) {
+        const uint64_t vd = dv0 + (uint64_t)(s * (kTileBytes >> 4));
+        const uint32_t d_tmem = tmem + 256 + qt * 128, a_tmem = tmem + qt * 128;
+        const uint32_t acc = accumulate ? 1u : 0u;
+        mma_ts_off<0 * 128>(d_tmem, a_tmem + 0, vd, idesc_pv, acc);
+        mma_ts_off<1 * 128>(d_tmem, a_tmem + 8, vd, idesc_pv, 1);
+        mma_ts_off<2 * 128>(d_tmem, a_tmem + 16, vd, idesc_pv, 1);
+        mma_ts_off<3 * 128>(d_tmem, a_tmem + 24, vd, idesc_pv, 1);
+        mma_ts_off<4 * 128>(d_tmem, a_tmem + 32, vd, idesc_pv, 1);
+        mma_ts_off<5 * 128>(d_tmem, a_tmem + 40, vd, idesc_pv, 1);
+        mma_ts_off<6 * 128>(d_tmem, a_tmem + 48, vd, idesc_pv, 1);
+        mma_ts_off<7 * 128>(d_tmem, a_tmem + 56, vd, idesc_pv, 1);
         tc_commit(cx.bar(kODone + qt));
+        }
+        __syncwarp();
       };
-      bool ok = cx.wait(kQFull, 0, 201) && cx.wait(kKFull + 0, 0, 202);
-      if (ok) {
-        tc_fence_after();
-        issue_qk(0, 0);
-        issue_qk(1, 0);
-        tc_commit(cx.bar(kKEmpty + 0));
-        if (n_rt == 1) tc_commit(cx.bar(kQCurDone));
-      }
-      for (int t = 0; ok && t < T; ++t) {
-        const int s = t & 1;
-        const uint32_t ph = (t >> 1) & 1;
-        const bool next = t + 1 < T;
-        const bool switch_next = next && (t + 1 == n_rt);
-        const int s1 = (t + 1) & 1;
-        const uint32_t ph1 = ((t + 1) >> 1) & 1;
-        if (!(ok = cx.wait(kVFull + s, ph, 203))) break;
-        if (!(ok = cx.wait(kPFull + 0, t & 1, 204))) break;
-        tc_fence_after();
-        issue_pv(0, t);
-        if (next && !switch_next) {
-          if (!(ok = cx.wait(kKFull + s1, ph1, 205))) break;
-          tc_fence_after();
-          issue_qk(0, t + 1);
-        }
-        if (!(ok = cx.wait(kPFull + 1, t & 1, 206))) break;
-        tc_fence_after();
-        issue_pv(1, t);
-        tc_commit(cx.bar(kVEmpty + s));
-        if (next) {
-          if (switch_next) {
-            if (!(ok = cx.wait(kQRotFull, 0, 207))) break;
-            if (!(ok = cx.wait(kKFull + s1, ph1, 208))) break;
-            tc_fence_after();
-            issue_qk(0, t + 1);
+      Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+      Segment sg;
+      int it = 0, nseg = 0;
+      bool ok = true;
+      while (ok && sch.next(sg)) {
+        const uint32_t sp = nseg & 1;
+        // last current-chunk tile of this segment (-1 if the segment starts in the cache): after its
+        // score MMAs nothing reads the unrotated query any more
+        const int t_lastcur = (sg.tb < n_rt) ? min(sg.te, n_rt) - 1 : -1;
+        if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, sp, 201)))) break;
+        {
+          const bool cached0 = sg.tb >= n_rt;
+          if (cached0) {
+            commit1(cx.bar(kQCurDone));
+            if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQRotFull, sp, 207)))) break;
           }
-          issue_qk(1, t + 1);
-          tc_commit(cx.bar(kKEmpty + s1));
-          if (t + 1 == n_rt - 1) tc_commit(cx.bar(kQCurDone));
+          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + (it & 1), (it >> 1) & 1, 202)))) break;
+          tc_fence_after();
+          issue_qk(0, it & 1, cached0);
+          issue_qk(1, it & 1, cached0);
+          commit1(cx.bar(kKEmpty + (it & 1)));
+          if (sg.tb == t_lastcur) commit1(cx.bar(kQCurDone));
         }
+        for (int t = sg.tb; t < sg.te; ++t, ++it) {
+          const int s = it & 1;
+          const uint32_t ph = (it >> 1) & 1;
+          const bool first = t == sg.tb;
+          const bool next = t + 1 < sg.te;
+          const bool switch_next = next && (t + 1 == n_rt);
+          const bool next_cached = t + 1 >= n_rt;
+          const int s1 = (it + 1) & 1;
+          const uint32_t ph1 = ((it + 1) >> 1) & 1;
+          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kVFull + s, ph, 203)))) break;
+          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kPFull + 0, it & 1, 204)))) break;
+          if (first && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kOFree + 0, sp ^ 1, 209)))) break;   // previous segment's O has been read out
+          tc_fence_after();
+          issue_pv(0, s, !first);
+          if (next && !switch_next) {
+            if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + s1, ph1, 205)))) break;
+            tc_fence_after();
+            issue_qk(0, s1, next_cached);
+          }
+          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kPFull + 1, it & 1, 206)))) break;
+          if (first && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kOFree + 1, sp ^ 1, 210)))) break;
+          tc_fence_after();
+          issue_pv(1, s, !first);
+          commit1(cx.bar(kVEmpty + s));
+          if (next) {
+            if (switch_next) {
+              if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQRotFull, sp, 207)))) break;
+              if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + s1, ph1, 208)))) break;
+              tc_fence_after();
+              issue_qk(0, s1, true);
+            }
+            issue_qk(1, s1, next_cached);
+            commit1(cx.bar(kKEmpty + s1));
+            if (t + 1 == t_lastcur) commit1(cx.bar(kQCurDone));
+          }
+        }
+        if (!ok) break;
+        commit1(cx.bar(kQEmpty));
+        ++nseg;
       }
       // everything issued so far must have retired before TMEM is freed
-      tc_commit(cx.bar(kDrain));
+      commit1(cx.bar(kDrain));
       cx.drain(kDrain, 0);
     }
   }
   } else if (warp < 12) {
     // ================= softmax groups =================
+    // Both groups work on every query tile: warp 4+q and warp 8+q share TMEM lanes 32q..32q+31 (one row per
+    // lane) and take columns [0,64) and [64,128) of that row's scores.  The two warps exchange their partial
+    // row maxima through shared memory (pair barrier), so a tile's softmax latency is that of 64 elements.
     setmaxnreg_inc<kRegsSoftmax>();
-    const int qt = (warp - 4) >> 2;
-    const int wq = warp & 3;
-    const int r_in_tile = wq * 32 + lane;
-    const int row = row0 + qt * kBlockM + r_in_tile;
+    const int half = (warp - 4) >> 2;                         // which 64 columns
+    const int wq = warp & 3;                                  // which 32 rows (TMEM lane quarter)
+    const int r128 = wq * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-    const uint32_t s_addr = tmem + lane_addr + qt * 128;
-    const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128;
     const float c_row = p.scale_log2;
-    float m = -INFINITY, l_cur = 0.f, l_cac = 0.f;
+    float* xmax = reinterpret_cast<float*>(smem + kOffXmax);
+    float* xl = reinterpret_cast<float*>(smem + kOffXl);
+    Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+    Segment sg;
+    int it = 0, nseg = 0;
+    uint32_t pair_phase = 0;                                  // pair barriers flip once per tile and once per epilogue
     bool ok = true;
-    for (int t = 0; t < T; ++t) {
-      const bool cached = t >= n_rt;
-      const int n_valid = cached ? min(kBlockN, p.n_cached - (t - n_rt) * kBlockN) : min(kBlockN, p.n_cur - t * kBlockN);
-      ok = __all_sync(0xFFFFFFFFu, cx.wait(kSFull + qt, t & 1, 301));
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t sr[128];                          // this row's 128 scores, then its 64 packed probabilities
+    while (ok && sch.next(sg)) {
+      float m[2] = {-INFINITY, -INFINITY}, l_cur[2] = {0.f, 0.f}, l_cac[2] = {0.f, 0.f};
+      uint32_t sr[64];                           // this thread's 64 scores, then its 32 packed probabilities
+      for (int t = sg.tb; ok && t < sg.te; ++t, ++it) {
+        const bool cached = t >= n_rt;
+        const int n_valid = (cached ? min(kBlockN, p.n_cached - (t - n_rt) * kBlockN) : min(kBlockN, p.n_cur - t * kBlockN)) - half * 64;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + 32 * c, sr + 32 * c);
-      tmem_wait_ld();
-      if (n_valid < kBlockN) {                   // ragged last tile of a segment
-#pragma unroll
-        for (int i = 0; i < 128; ++i)
-          if (i >= n_valid) sr[i] = 0xFF800000u;  // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < 128; i += 4) {
-        mx0 = max3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
-        mx1 = max3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
-      }
-      const float m_new = fmaxf(m, fmaxf(mx0, mx1) * c_row);
-      if (__any_sync(0xFFFFFFFFu, m_new - m > kRescaleThreshold)) {
-        if (t > 0) {
-          ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (t - 1) & 1, 302));
+        for (int qt = 0; qt < 2; ++qt) {
+          const int r256 = qt * kBlockM + r128;
+          const uint32_t s_addr = tmem + lane_addr + qt * 128 + half * 64;
+          const uint32_t p_addr = tmem + lane_addr + qt * 128 + half * 32;
+          const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128 + half * 64;
+          ok = __all_sync(0xFFFFFFFFu, cx.wait(kSFull + qt, it & 1, 301));
           if (!ok) break;
           tc_fence_after();
-          const float f = ex2(m - m_new);
+          tmem_ld32(s_addr, sr);
+          tmem_ld32(s_addr + 32, sr + 32);
+          tmem_wait_ld();
+          if (n_valid < 64) {                      // ragged last tile of the current chunk or of the cache
+#pragma unroll
+            for (int i = 0; i < 64; ++i)
+              if (i >= n_valid) sr[i] = 0xFF800000u;  // -inf
+          }
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int i = 0; i < 64; i += 8) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) mx[c] = max3(mx[c], __uint_as_float(sr[i + 2 * c]), __uint_as_float(sr[i + 2 * c + 1]));
+          }
+          const float mine = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          xmax[half * 256 + r256] = mine;
+          tc_fence_before();
+          mbar_arrive(cx.bar(kPair + qt * 4 + wq));
+          ok = __all_sync(0xFFFFFFFFu, cx.wait(kPair + qt * 4 + wq, pair_phase, 304));
+          if (!ok) break;
+          tc_fence_after();
+          const float m_new = fmaxf(m[qt], fmaxf(mine, xmax[(half ^ 1) * 256 + r256]) * c_row);
+          if (__any_sync(0xFFFFFFFFu, m_new - m[qt] > kRescaleThreshold)) {
+            if (t > sg.tb) {
+              ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (it - 1) & 1, 302));
+              if (!ok) break;
+              tc_fence_after();
+              const float f = ex2(m[qt] - m_new);
 #pragma unroll 1
-          for (int c = 0; c < 8; ++c) {
-            uint32_t r[16];
-            tmem_ld16(o_addr + 16 * c, r);
-            tmem_wait_ld();
+              for (int c = 0; c < 4; ++c) {
+                uint32_t r[16];
+                tmem_ld16(o_addr + 16 * c, r);
+                tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-            tmem_st16(o_addr + 16 * c, r);
+                for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+                tmem_st16(o_addr + 16 * c, r);
+              }
+              l_cur[qt] *= f; l_cac[qt] *= f;
+            }
+            m[qt] = m_new;
           }
-          l_cur *= f; l_cac *= f;
+          const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m[qt], -m[qt]);
+          float2 sum2 = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int i = 0; i < 64; i += 2) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), c2, nm2);
+            // the MUFU pipe (16 ex2 per clock per SM) is the scarcer unit: a fixed share of the pairs goes to the FMA pipe
+            const float2 pr = ((kFmaPipePairs >> (i >> 1)) & 1u) ? exp2_fma_pipe(x) : make_float2(ex2(x.x), ex2(x.y));
+            sum2 = __fadd2_rn(sum2, pr);
+            sr[i >> 1] = cvt_bf16x2(pr.x, pr.y);
+          }
+          tmem_st32(p_addr, sr);
+          if (cached) l_cac[qt] += sum2.x + sum2.y; else l_cur[qt] += sum2.x + sum2.y;
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(cx.bar(kPFull + qt));
         }
-        m = m_new;
+        pair_phase ^= 1;
       }
-      const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m, -m);
-      float2 sum2 = make_float2(0.f, 0.f);
+      if (!ok) break;
+      // ---- segment epilogue: read O out of TMEM, release it, combine the two column halves' row sums ----
+      const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
+      const bool whole = sg.tb == 0 && sg.te == T;
+      float* slot = p.partial + (size_t)(2 * blockIdx.x + (nseg > 0 ? 1 : 0)) * kSlotFloats;   // partial segments only
 #pragma unroll
-      for (int i = 0; i < 128; i += 2) {
-        const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), c2, nm2);
-        const float p0 = ex2(x.x), p1 = ex2(x.y);
-        sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
-        sr[i >> 1] = cvt_bf16x2(p0, p1);
-      }
-      tmem_st32(s_addr, sr);
-      tmem_st32(s_addr + 32, sr + 32);
-      if (cached) l_cac += sum2.x + sum2.y; else l_cur += sum2.x + sum2.y;
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(cx.bar(kPFull + qt));
-    }
-    if (ok) ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (T - 1) & 1, 303));
-    if (ok) {
-      tc_fence_after();
-      const float l = l_cur + l_cac;
-      const float inv = 1.0f / l;
-      uint16_t* dst = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(o_addr + 32 * c, r);
+      for (int qt = 0; qt < 2; ++qt) {
+        const int r256 = qt * kBlockM + r128;
+        const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128 + half * 64;
+        ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (it - 1) & 1, 303));
+        if (!ok) break;
+        tc_fence_after();
+        tmem_ld32(o_addr, sr);
+        tmem_ld32(o_addr + 32, sr + 32);
         tmem_wait_ld();
-        if (row < p.m_tokens) {
+        tc_fence_before();
+        mbar_arrive(cx.bar(kOFree + qt));
+        xl[(half * 256 + r256) * 2] = l_cur[qt];
+        xl[(half * 256 + r256) * 2 + 1] = l_cac[qt];
+        mbar_arrive(cx.bar(kPair + qt * 4 + wq));
+        ok = __all_sync(0xFFFFFFFFu, cx.wait(kPair + qt * 4 + wq, pair_phase, 305));
+        if (!ok) break;
+        const float lc = l_cur[qt] + xl[((half ^ 1) * 256 + r256) * 2];
+        const float la = l_cac[qt] + xl[((half ^ 1) * 256 + r256) * 2 + 1];
+        const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
+        if (whole) {
+          if (row < p.m_tokens) {
+            const float l = lc + la;
+            const float inv = 1.0f / l;
+            uint16_t* dst = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + half * 64;
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 v;
-            v.x = pack_bf16x2(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-            v.y = pack_bf16x2(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-            v.z = pack_bf16x2(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-            v.w = pack_bf16x2(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + 32 * c + i) = v;
+            for (int i = 0; i < 64; i += 8) {
+              uint4 v;
+              v.x = cvt_bf16x2(__uint_as_float(sr[i]) * inv, __uint_as_float(sr[i + 1]) * inv);
+              v.y = cvt_bf16x2(__uint_as_float(sr[i + 2]) * inv, __uint_as_float(sr[i + 3]) * inv);
+              v.z = cvt_bf16x2(__uint_as_float(sr[i + 4]) * inv, __uint_as_float(sr[i + 5]) * inv);
+              v.w = cvt_bf16x2(__uint_as_float(sr[i + 6]) * inv, __uint_as_float(sr[i + 7]) * inv);
+              *reinterpret_cast<uint4*>(dst + i) = v;
+            }
+            if (half == 0) {
+              const int64_t idx = (int64_t)bh * p.m_tokens + row;
+              if (p.lse) p.lse[idx] = (m[qt] + log2f(l)) * 0.6931471805599453f;
+              if (p.cached_mass) p.cached_mass[idx] = la * inv;
+            }
+          }
+        } else {
+          float4* orow = reinterpret_cast<float4*>(slot + (size_t)r256 * kD + half * 64);
+#pragma unroll
+          for (int i = 0; i < 64; i += 4)
+            orow[i >> 2] = make_float4(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1]), __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+          if (half == 0) {
+            slot[256 * kD + r256] = m[qt];
+            slot[256 * kD + 256 + r256] = lc;
+            slot[256 * kD + 512 + r256] = la;
           }
         }
       }
-      if (row < p.m_tokens) {
-        const int64_t idx = (int64_t)bh * p.m_tokens + row;
-        if (p.lse) p.lse[idx] = (m + log2f(l)) * 0.6931471805599453f;
-        if (p.cached_mass) p.cached_mass[idx] = l_cac * inv;
-      }
+      pair_phase ^= 1;
+      ++nseg;
     }
     tc_fence_before();
   } else {
     // ================= dequant + query rotation =================
     setmaxnreg_dec<kRegsDequant>();
     const int dt = tid - 12 * 32;          // 0..127: the key of the tile this thread expands
-    const int64_t tok0 = (int64_t)bh * p.capacity + p.cache_begin;
-    Raw<BITS> rk, rv;
-    if (n_ct > 0) {
-      const bool valid = dt < p.n_cached;
-      load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + dt, valid);
-      load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + dt, valid);
-    }
+    Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+    Segment sg;
+    int it = 0, nseg = 0;
     bool ok = true;
-    for (int t = 0; t < T; ++t) {
-      const int s = t & 1;
-      const uint32_t ph = (t >> 1) & 1;
-      const int ct = t - n_rt;
-      ok = __all_sync(0xFFFFFFFFu, cx.wait(kKEmpty + s, ph ^ 1, 401));
-      if (!ok) break;
-      if (ct >= 0) {
-        dequant_keys<BITS, GROUP>(rk, smem + kOffK + s * kTileBytes, dt);
-        if (p.correction) {   // B_extra row: step_j^2, exact in BF16
-          const float d0 = raw_step<BITS>(rk, 0), d1 = raw_step<BITS>(rk, 1), d2 = raw_step<BITS>(rk, 2), d3 = raw_step<BITS>(rk, 3);
-          const uint32_t b01 = pack_bf16x2(d0 * d0, G > 1 ? d1 * d1 : 0.f), b23 = pack_bf16x2(G > 2 ? d2 * d2 : 0.f, G > 3 ? d3 * d3 : 0.f);
-          // columns 0..3 meet the high parts of A_extra, columns 4..7 the low parts
-          *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(dt, 0)) = make_uint4(b01, b23, b01, b23);
-        }
-        fence_proxy_async_smem();
-        if (ct + 1 < n_ct) {
-          const int k1 = (ct + 1) * kBlockN + dt;
-          load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k1, k1 < p.n_cached);
-        }
+    Raw<BITS> rk, rv;
+    while (ok && sch.next(sg)) {
+      const int bh = sg.unit / p.q_blocks;
+      const int64_t tok0 = (int64_t)bh * p.capacity + p.cache_begin;
+      const int t_rot = max(sg.tb, n_rt);          // first cached tile of the segment: the query is rotated there
+      if (sg.te > n_rt) {
+        const int k0 = (t_rot - n_rt) * kBlockN + dt;
+        load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k0, k0 < p.n_cached);
+        load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k0, k0 < p.n_cached);
       }
-      mbar_arrive(cx.bar(kKFull + s));
-      if (ct == 0) {
-        // ---- rotate the query tile in place; per-group squared norms -> A_extra ----
-        ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, 0, 402) && cx.wait(kQCurDone, 0, 403));
+      for (int t = sg.tb; t < sg.te; ++t, ++it) {
+        const int s = it & 1;
+        const uint32_t ph = (it >> 1) & 1;
+        const int ct = t - n_rt;
+        const int k1 = (ct + 1) * kBlockN + dt;    // this thread's key in the next tile
+        ok = __all_sync(0xFFFFFFFFu, cx.wait(kKEmpty + s, ph ^ 1, 401));
         if (!ok) break;
-        const int l16 = lane & 15, rsub = lane >> 4;
-        constexpr int lanes_per_group = GROUP / 8;
-        float sgn[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) sgn[e] = (p.rotate && p.signs) ? (float)p.signs[l16 * 8 + e] : 1.0f;
-        for (int pass = 0; pass < 32; ++pass) {
-          const int qrow = pass * 8 + (warp - 12) * 2 + rsub;     // 0..255
-          const int qt = qrow >> 7, rr = qrow & 127;
-          uint8_t* qtile = smem + kOffQ + qt * kTileBytes;
-          const uint4 raw = *reinterpret_cast<const uint4*>(qtile + sw128_offset(rr, l16));
-          float x[8];
-          x[0] = bf16_bits_to_f32(raw.x & 0xFFFFu); x[1] = bf16_bits_to_f32(raw.x >> 16);
-          x[2] = bf16_bits_to_f32(raw.y & 0xFFFFu); x[3] = bf16_bits_to_f32(raw.y >> 16);
-          x[4] = bf16_bits_to_f32(raw.z & 0xFFFFu); x[5] = bf16_bits_to_f32(raw.z >> 16);
-          x[6] = bf16_bits_to_f32(raw.w & 0xFFFFu); x[7] = bf16_bits_to_f32(raw.w >> 16);
-          if (p.rotate) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] *= sgn[e];
-#pragma unroll
-            for (int hh = 1; hh < 8; hh *= 2)
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                if ((i & hh) == 0) { const float a = x[i], c = x[i + hh]; x[i] = a + c; x[i + hh] = a - c; }
-#pragma unroll
-            for (int lm = 1; lm < 16; lm *= 2)
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
-                x[e] = (l16 & lm) ? (o - x[e]) : (x[e] + o);
-              }
-#pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] *= 0.08838834764831845f;
+        if (ct >= 0) {
+          dequant_keys<BITS, GROUP>(rk, smem + kOffK + s * kTileBytes, dt);
+          if (p.correction) {   // B_extra row: step_j^2, exact in BF16
+            const float d0 = raw_step<BITS>(rk, 0), d1 = raw_step<BITS>(rk, 1), d2 = raw_step<BITS>(rk, 2), d3 = raw_step<BITS>(rk, 3);
+            const uint32_t b01 = pack_bf16x2(d0 * d0, G > 1 ? d1 * d1 : 0.f), b23 = pack_bf16x2(G > 2 ? d2 * d2 : 0.f, G > 3 ? d3 * d3 : 0.f);
+            // columns 0..3 meet the high parts of A_extra, columns 4..7 the low parts
+            *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(dt, 0)) = make_uint4(b01, b23, b01, b23);
           }
-          float nu = 0.f;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) nu += x[e] * x[e];
-          for (int off = 1; off < lanes_per_group; off *= 2) nu += __shfl_xor_sync(0xFFFFFFFFu, nu, off);
-          if ((l16 % lanes_per_group) == 0) {
-            const int j = l16 / lanes_per_group;
-            // -(sigma/24) nu as a BF16 high part plus a BF16 low part (columns j and 4 + j)
-            const float a = p.ax_coef * nu;
-            const uint32_t hi = f32_to_bf16_bits(a);
-            uint8_t* ax = smem + kOffAx + qt * kXBytes + xtile_offset(rr, 0);
-            *reinterpret_cast<uint16_t*>(ax + 2 * j) = (uint16_t)hi;
-            *reinterpret_cast<uint16_t*>(ax + 8 + 2 * j) = (uint16_t)f32_to_bf16_bits(a - bf16_bits_to_f32(hi));
-          }
-          float y[8];
-          if constexpr (BITS == 2) {
-            // physical column 16w + 2i + hsel <- channel 16w + i + 8*hsel: even lanes own the low half
-            // of a 16-channel word, odd lanes the high half; swap four values with the neighbour
-            const bool odd = l16 & 1;
-            float rcv[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) rcv[i] = __shfl_xor_sync(0xFFFFFFFFu, odd ? x[i] : x[4 + i], 1);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              y[2 * i] = odd ? rcv[i] : x[i];
-              y[2 * i + 1] = odd ? x[4 + i] : rcv[i];
-            }
-          } else {
-            // physical column 8w + 2i + hsel <- channel 8w + i + 4*hsel
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { y[2 * i] = x[i]; y[2 * i + 1] = x[4 + i]; }
-          }
-          *reinterpret_cast<uint4*>(qtile + sw128_offset(rr, l16)) =
-              make_uint4(pack_f16x2_sat(y[0], y[1]), pack_f16x2_sat(y[2], y[3]), pack_f16x2_sat(y[4], y[5]), pack_f16x2_sat(y[6], y[7]));
+          fence_proxy_async_smem();
+          if (t + 1 < sg.te) load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k1, k1 < p.n_cached);
         }
-        fence_proxy_async_smem();
-        mbar_arrive(cx.bar(kQRotFull));
+        mbar_arrive(cx.bar(kKFull + s));
+        if (t == t_rot) {
+          // ---- rotate the query tile in place; per-group squared norms -> A_extra ----
+          ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, nseg & 1, 402) && cx.wait(kQCurDone, nseg & 1, 403));
+          if (!ok) break;
+          rotate_query<BITS, GROUP>(smem, p, warp, lane);
+          fence_proxy_async_smem();
+          mbar_arrive(cx.bar(kQRotFull));
+        }
+        ok = __all_sync(0xFFFFFFFFu, cx.wait(kVEmpty + s, ph ^ 1, 404));
+        if (!ok) break;
+        if (ct >= 0) {
+          dequant_values<BITS, GROUP>(rv, smem + kOffV + s * kTileBytes, dt);
+          fence_proxy_async_smem();
+          if (t + 1 < sg.te) load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k1, k1 < p.n_cached);
+        }
+        mbar_arrive(cx.bar(kVFull + s));
       }
-      ok = __all_sync(0xFFFFFFFFu, cx.wait(kVEmpty + s, ph ^ 1, 404));
       if (!ok) break;
-      if (ct >= 0) {
-        dequant_values<BITS, GROUP>(rv, smem + kOffV + s * kTileBytes, dt);
-        fence_proxy_async_smem();
-        if (ct + 1 < n_ct) {
-          const int k1 = (ct + 1) * kBlockN + dt;
-          load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k1, k1 < p.n_cached);
-        }
-      }
-      mbar_arrive(cx.bar(kVFull + s));
+      if (sg.te <= n_rt) mbar_arrive(cx.bar(kQRotFull));   // no rotation in this segment: keep the phase count in step
+      ++nseg;
     }
   }
 
@@ -682,6 +859,57 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
+  }
+}
+
+// Combines the partial results of every unit whose key tiles were split over several CTAs.
+// grid (n_units, 32): a block handles 8 rows x 128 columns; thread = (row, 8-column group).
+__global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_ctas) {
+  const int unit = blockIdx.x;
+  const int T = p.tiles;
+  const long long W = (long long)p.n_units * T;
+  const long long g_lo = (long long)unit * T, g_hi = g_lo + T;
+  auto start = [&](long long c) { return W * c / n_ctas; };
+  auto owner = [&](long long g) {
+    long long c = g * n_ctas / W;
+    while (c + 1 < n_ctas && start(c + 1) <= g) ++c;
+    while (c > 0 && start(c) > g) --c;
+    return (int)c;
+  };
+  const int c_first = owner(g_lo), c_last = owner(g_hi - 1);
+  if (c_first == c_last) return;                       // the unit was computed whole by one CTA
+  const int r256 = blockIdx.y * 8 + (threadIdx.x >> 4);
+  const int cg = threadIdx.x & 15;
+  const int bh = unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
+  const int row = (unit - bh * p.q_blocks) * 256 + r256;
+  if (row >= p.m_tokens) return;
+  float m = -INFINITY;
+  for (int c = c_first; c <= c_last; ++c) {
+    const int slot = 2 * c + ((int)(start(c) / T) == unit ? 0 : 1);
+    m = fmaxf(m, p.partial[(size_t)slot * kSlotFloats + 256 * kD + r256]);
+  }
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float l_cur = 0.f, l_cac = 0.f;
+  for (int c = c_first; c <= c_last; ++c) {
+    const int slot = 2 * c + ((int)(start(c) / T) == unit ? 0 : 1);
+    const float* sl = p.partial + (size_t)slot * kSlotFloats;
+    const float f = exp2f(sl[256 * kD + r256] - m);
+    l_cur += f * sl[256 * kD + 256 + r256];
+    l_cac += f * sl[256 * kD + 512 + r256];
+    const float4 a0 = *reinterpret_cast<const float4*>(sl + (size_t)r256 * kD + cg * 8);
+    const float4 a1 = *reinterpret_cast<const float4*>(sl + (size_t)r256 * kD + cg * 8 + 4);
+    acc[0] += f * a0.x; acc[1] += f * a0.y; acc[2] += f * a0.z; acc[3] += f * a0.w;
+    acc[4] += f * a1.x; acc[5] += f * a1.y; acc[6] += f * a1.z; acc[7] += f * a1.w;
+  }
+  const float l = l_cur + l_cac, inv = 1.0f / l;
+  uint4 v;
+  v.x = cvt_bf16x2(acc[0] * inv, acc[1] * inv); v.y = cvt_bf16x2(acc[2] * inv, acc[3] * inv);
+  v.z = cvt_bf16x2(acc[4] * inv, acc[5] * inv); v.w = cvt_bf16x2(acc[6] * inv, acc[7] * inv);
+  *reinterpret_cast<uint4*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + cg * 8) = v;
+  if (cg == 0) {
+    const int64_t idx = (int64_t)bh * p.m_tokens + row;
+    if (p.lse) p.lse[idx] = (m + log2f(l)) * 0.6931471805599453f;
+    if (p.cached_mass) p.cached_mass[idx] = l_cac * inv;
   }
 }
 
@@ -723,6 +951,32 @@ int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, kvq_strides s
   return KVQ_OK;
 }
 
+int num_sms() {
+  static int cached = 0;
+  if (!cached) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+    cached = n;
+  }
+  return cached;
+}
+
+// Grid policy.  With at least half as many units as SMs every CTA takes one whole unit (no partial results,
+// the hardware scheduler balances the waves; measured faster than splitting on the chunk-sized workloads).
+// With fewer units (short query chunk, long cache) the n_units * tiles key-tile steps are cut into equal
+// contiguous ranges, one per SM, each at least ~4 tiles long, and split units are merged afterwards.
+int grid_ctas(int64_t n_units, int64_t tiles) {
+  const int sms = num_sms();
+  if (2 * n_units >= sms) return (int)n_units;
+  const int64_t W = n_units * tiles;
+  int64_t c = W / 4;
+  if (c < n_units) c = n_units;
+  if (c > sms) c = sms;
+  if (c > W) c = W;
+  return (int)(c < 1 ? 1 : c);
+}
+
 template <int BITS, int GROUP>
 int launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TParams& p, dim3 grid, cudaStream_t st) {
   static bool configured = false;
@@ -732,16 +986,33 @@ int launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, 
   }
   attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
   KVQ_CUDA_TRY(cudaGetLastError());
+  if ((int)grid.x != p.n_units) {   // units were split over CTAs: combine their partial results
+    attn_merge_kernel<<<dim3((unsigned)p.n_units, 32), 128, 0, st>>>(p, (int)grid.x);
+    KVQ_CUDA_TRY(cudaGetLastError());
+  }
   return KVQ_OK;
 }
 
 }  // namespace
 
 bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur) {
-  return d->head_dim == kD && m_tokens >= 1 && n_cur >= 1 && (int64_t)d->batch * d->heads <= 65535;
+  return d->head_dim == kD && m_tokens >= 1 && n_cur >= 1;
 }
 
-size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc*, int64_t, int64_t, int64_t) { return 0; }
+static void schedule_shape(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur,
+                           int64_t* q_blocks, int64_t* n_units, int64_t* tiles) {
+  *q_blocks = (m_tokens + 2 * kBlockM - 1) / (2 * kBlockM);
+  *n_units = (int64_t)d->batch * d->heads * *q_blocks;
+  *tiles = (n_cur + kBlockN - 1) / kBlockN + (cache_len + kBlockN - 1) / kBlockN;
+}
+
+size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur) {
+  if (m_tokens <= 0) return 0;
+  int64_t qb, nu, tiles;
+  schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
+  const int c = grid_ctas(nu, tiles);
+  return c != nu ? (size_t)c * 2 * kSlotFloats * sizeof(float) : 0;
+}
 
 int launch_attn_tcgen05(const AttnArgs& a) {
   const kvq_cache_desc* d = a.desc;
@@ -765,7 +1036,12 @@ int launch_attn_tcgen05(const AttnArgs& a) {
   p.scale_log2 = a.softmax_scale * kLog2e;
   p.ax_coef = -a.softmax_scale / 24.0f;
   p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
-  dim3 grid((unsigned)((a.m_tokens + 2 * kBlockM - 1) / (2 * kBlockM)), (unsigned)((int64_t)d->batch * d->heads));
+  int64_t qb, nu, tiles;
+  schedule_shape(d, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
+  if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
+  p.partial = static_cast<float*>(a.workspace);
+  dim3 grid((unsigned)grid_ctas(nu, tiles));
   if (d->bits == 2) {
     if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
     if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);

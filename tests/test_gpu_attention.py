@@ -90,6 +90,27 @@ def test_ragged_shapes_all_formats(B, d, bits, group):
     _compare(B, g, o, n, q, kc, vc, T.sigma_of(d), sel)
 
 
+def test_short_chunk_long_cache_is_split_over_ctas(B):
+    """Few (batch, head, query block) units and a long cache: the tcgen05 kernel cuts the key tiles of a unit
+    over several CTAs and merges their partial results (needs the workspace)."""
+    w = inputs.Workload("split", 320, 1, 2, 128, 200, 0, 2, 64, 0, k_outliers=2, k_outlier_scale=4.0)
+    g, o, n, sel = _build(B, w, 9, tokens=1111, cap=10112)
+    assert n == 9999
+    q, kc, vc = inputs.make_chunk(w, 20)
+    assert B.kvq_attn_workspace_bytes(g, n, 200, 200, B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05) > 0
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(128), sel)
+    # a missing workspace is refused on the host
+    import ctypes as C
+    d = g.desc
+    s = B.kvq_strides(q.shape[1] * 200 * 128, 200 * 128, 128)
+    qd = T.to_dev(q)
+    out = torch.empty_like(qd)
+    rc = B.lib.kvq_attn_corrected(C.byref(d), 0, n, qd.data_ptr(), s, qd.data_ptr(), qd.data_ptr(), s, 200, 200,
+                                  out.data_ptr(), s, 0.088, B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05,
+                                  None, None, None, 0, None, None)
+    assert rc == B.KVQ_ERR_WORKSPACE
+
+
 def test_empty_cache_is_plain_attention(B):
     w = inputs.Workload("empty", 300, 1, 2, 128, 150, 0, 2, 64, 0)
     g = B.Cache(1, 2, 128, 2, 64, 128)
