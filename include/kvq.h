@@ -164,6 +164,40 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
                        int32_t* status_word, kvq_stream_t stream);
 
 /*
+ * kvq_attn_corrected for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a deployment variant of the call above, same arithmetic, same outputs.)
+ *
+ * Who needs it: code that must not call cudaMalloc — a serving process that has handed all device memory
+ * to its framework's pool, a plug-in that only ever receives input and output pointers, anything that runs
+ * where an allocation would synchronise the device or is forbidden.  kvq_attn_corrected needs a caller
+ * workspace when it splits the key tiles of a unit over several CTAs (few query rows, long cache); this
+ * entry point keeps those partial results in a scratch buffer that is part of the library image instead:
+ * 64 slots of 134 144 bytes = 8 585 216 bytes of device memory on every GPU that loads libkvq.so, held
+ * until the process exits.  It calls no allocating routine of CUDA or of any other library.
+ *
+ * Limits: head_dim 128 only (the tcgen05 kernel; no kernel-selection flags).  A problem whose units
+ * (batch * heads * ceil(m_tokens / 256)) are fewer than half the SMs is split, on at most 32 CTAs, and may
+ * then have at most 32 units: more returns KVQ_ERR_WORKSPACE.  Larger problems are not split, use no
+ * scratch and are accepted at any size.
+ *
+ * The first call on a device looks up the buffer's device address (cudaGetSymbolAddress, with that device
+ * current) and remembers it; make that first call outside any stream capture.
+ * All calls on a device share the one buffer and it keeps the previous call's contents.  Nothing in it has
+ * to start at zero (every slot is written in full before it is read), so no clearing is done; but two calls
+ * whose kernels overlap on the GPU (different streams, no ordering between them) race on it: order them.
+ *
+ * Arguments, outputs and the other error codes are those of kvq_attn_corrected, without the workspace.
+ */
+int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
+                                      const void* q, kvq_strides q_strides,
+                                      const void* k_cur, const void* v_cur, kvq_strides kv_strides,
+                                      int64_t m_tokens, int64_t n_cur,
+                                      void* out_bf16, kvq_strides o_strides,
+                                      float softmax_scale, uint32_t flags,
+                                      float* lse_out, float* cached_mass_out,
+                                      int32_t* status_word, kvq_stream_t stream);
+
+/*
  * Test aid: expand the packed codes of cache tokens [begin, begin + n) to one byte per element,
  * out_codes device u8 [batch, heads, n, head_dim], in canonical channel order (the order of
  * Eq. (1)'s vector x).  which: 0 = keys, 1 = values.

@@ -64,6 +64,12 @@ def _load():
         C.c_void_p, kvq_strides, C.c_void_p, C.c_void_p, kvq_strides,
         C.c_int64, C.c_int64, C.c_void_p, kvq_strides,
         C.c_float, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    lib.kvq_attn_corrected_static_scratch.restype = C.c_int
+    lib.kvq_attn_corrected_static_scratch.argtypes = [
+        C.POINTER(kvq_cache_desc), C.c_int64, C.c_int64,
+        C.c_void_p, kvq_strides, C.c_void_p, C.c_void_p, kvq_strides,
+        C.c_int64, C.c_int64, C.c_void_p, kvq_strides,
+        C.c_float, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.kvq_unpack_codes.restype = C.c_int
     lib.kvq_unpack_codes.argtypes = [C.POINTER(kvq_cache_desc), C.c_int, C.c_int64, C.c_int64,
                                      C.c_void_p, C.c_void_p]
@@ -184,6 +190,25 @@ def kvq_attn_corrected(cache: Cache, q, k_cur, v_cur, softmax_scale, flags=KVQ_C
         _strides(k_cur), m, n_cur, out.data_ptr(), _strides(out), float(softmax_scale), flags,
         _ptr(lse), _ptr(cached_mass), _ptr(ws), ws.numel() if ws is not None else 0, _ptr(status_word), _stream()),
         "kvq_attn_corrected")
+    return out
+
+
+def kvq_attn_corrected_static_scratch(cache: Cache, q, k_cur, v_cur, softmax_scale, flags=KVQ_CORRECTION_ON,
+                                      cache_begin=0, cache_len=None, out=None, lse=None, cached_mass=None,
+                                      status_word=None):
+    """kvq_attn_corrected without a workspace: split units keep their partial results in the scratch buffer
+    built into the library.  `out` must be given by callers that may not allocate; it is allocated here only
+    as a convenience when omitted."""
+    for t in (q, k_cur, v_cur):
+        assert t.dtype == torch.bfloat16 and t.is_cuda
+    assert k_cur.shape == v_cur.shape and k_cur.stride() == v_cur.stride()
+    n_cache = cache.length - cache_begin if cache_len is None else cache_len
+    if out is None:
+        out = torch.empty_like(q, memory_format=torch.contiguous_format)
+    _check(lib.kvq_attn_corrected_static_scratch(
+        C.byref(cache.desc), cache_begin, n_cache, q.data_ptr(), _strides(q), k_cur.data_ptr(), v_cur.data_ptr(),
+        _strides(k_cur), q.shape[2], k_cur.shape[2], out.data_ptr(), _strides(out), float(softmax_scale), flags,
+        _ptr(lse), _ptr(cached_mass), _ptr(status_word), _stream()), "kvq_attn_corrected_static_scratch")
     return out
 
 

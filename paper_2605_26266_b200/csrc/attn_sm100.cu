@@ -1052,4 +1052,80 @@ int launch_attn_tcgen05(const AttnArgs& a) {
   return launch<4, 128>(mq, mk, mv, p, grid, a.stream);
 }
 
+
+// ---- variant with built-in scratch ---------------------------------------------------------------
+//
+// Some callers may not allocate device memory at all (an inference server that hands its whole memory pool
+// to a framework allocator up front, code running while a CUDA graph is being captured, a plug-in that is
+// only given input and output pointers).  For them the split-unit path can run on a scratch buffer that is
+// part of the library image: every GPU that loads libkvq.so carries these 8.2 MiB until the process exits.
+constexpr int kStaticMaxCtas = 32;                         // split problems run on at most this many CTAs
+constexpr int kStaticSlots = 2 * kStaticMaxCtas;           // two partial results per CTA
+static __device__ __align__(256) float g_static_scratch[(size_t)kStaticSlots * kSlotFloats];
+
+// The array's name is only a host-side handle; the device address has to be asked for, once per device,
+// with that device current.
+static int static_scratch_ptr(float** out) {
+  constexpr int kMaxDevices = 64;
+  static float* ptrs[kMaxDevices] = {};
+  int dev = 0;
+  KVQ_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return KVQ_ERR_UNSUPPORTED;
+  if (!ptrs[dev]) {
+    void* p = nullptr;
+    KVQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (!p) return record_cuda_error(cudaErrorInvalidSymbol);
+    ptrs[dev] = static_cast<float*>(p);
+  }
+  *out = ptrs[dev];
+  return KVQ_OK;
+}
+
+int launch_attn_tcgen05_static(const AttnArgs& a) {
+  const kvq_cache_desc* d = a.desc;
+  int64_t qb, nu, tiles;
+  schedule_shape(d, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
+  if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  int ctas = grid_ctas(nu, tiles);
+  float* scratch = nullptr;
+  if (ctas != nu) {                                        // units are split: partial results need the scratch
+    if (nu > kStaticMaxCtas) return KVQ_ERR_WORKSPACE;     // stated maximum: 32 units when splitting
+    if (ctas > kStaticMaxCtas) ctas = kStaticMaxCtas;
+    if (ctas < nu) ctas = (int)nu;
+    const int r = static_scratch_ptr(&scratch);
+    if (r != KVQ_OK) return r;
+  }
+  EncodeTiledFn enc;
+  int r = get_encode_fn(&enc);
+  if (r != KVQ_OK) return r;
+  CUtensorMap mq, mk, mv;
+  if ((r = make_map(enc, &mq, a.q, a.qs, a.m_tokens, d->heads, d->batch)) != KVQ_OK) return r;
+  if ((r = make_map(enc, &mk, a.k_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
+  if ((r = make_map(enc, &mv, a.v_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
+  TParams p;
+  p.out = static_cast<uint16_t*>(a.out); p.o_sb = a.os.b; p.o_sh = a.os.h; p.o_st = a.os.t;
+  p.k_codes = static_cast<const uint8_t*>(d->k_codes); p.v_codes = static_cast<const uint8_t*>(d->v_codes);
+  p.k_scale = static_cast<const uint8_t*>(d->k_scale); p.v_scale = static_cast<const uint8_t*>(d->v_scale);
+  p.k_zero = static_cast<const uint16_t*>(d->k_zero); p.v_zero = static_cast<const uint16_t*>(d->v_zero);
+  p.signs = d->signs;
+  p.capacity = d->capacity; p.cache_begin = a.cache_begin;
+  p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
+  p.correction = (a.flags & KVQ_CORRECTION_ON) ? 1 : 0;
+  p.m_tokens = (int)a.m_tokens; p.n_cached = (int)a.cache_len; p.n_cur = (int)a.n_cur;
+  p.scale_log2 = a.softmax_scale * kLog2e;
+  p.ax_coef = -a.softmax_scale / 24.0f;
+  p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
+  p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
+  p.partial = scratch;
+  dim3 grid((unsigned)ctas);
+  if (d->bits == 2) {
+    if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
+    if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);
+    return launch<2, 128>(mq, mk, mv, p, grid, a.stream);
+  }
+  if (d->group == 32) return launch<4, 32>(mq, mk, mv, p, grid, a.stream);
+  if (d->group == 64) return launch<4, 64>(mq, mk, mv, p, grid, a.stream);
+  return launch<4, 128>(mq, mk, mv, p, grid, a.stream);
+}
+
 }  // namespace kvq

@@ -160,6 +160,32 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   return tc ? launch_attn_tcgen05(a) : launch_attn_mma_sync(a);
 }
 
+int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
+                                      const void* q, kvq_strides q_strides, const void* k_cur, const void* v_cur,
+                                      kvq_strides kv_strides, int64_t m_tokens, int64_t n_cur, void* out_bf16,
+                                      kvq_strides o_strides, float softmax_scale, uint32_t flags, float* lse_out,
+                                      float* cached_mass_out, int32_t* status_word, kvq_stream_t stream) {
+  if (flags & KVQ_KERNEL_MASK) return KVQ_ERR_INVALID_ARG;      // this entry point has one kernel only
+  int r = check_attn_args(desc, cache_begin, cache_len, m_tokens, n_cur, flags);
+  if (r != KVQ_OK) return r;
+  if ((r = check_desc(desc)) != KVQ_OK) return r;
+  if ((r = check_tensor(q, q_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(k_cur, kv_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
+  if (!attn_tcgen05_supports(desc, m_tokens, n_cur)) return KVQ_ERR_UNSUPPORTED;
+  if (m_tokens == 0) return KVQ_OK;
+  AttnArgs a;
+  a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;
+  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides;
+  a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out_bf16; a.os = o_strides;
+  a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse_out; a.cached_mass = cached_mass_out;
+  a.workspace = nullptr; a.workspace_bytes = 0; a.status_word = status_word;
+  a.stream = (cudaStream_t)stream;
+  return launch_attn_tcgen05_static(a);
+}
+
 int kvq_unpack_codes(const kvq_cache_desc* desc, int which, int64_t begin, int64_t n,
                      uint8_t* out_codes, kvq_stream_t stream) {
   int r = check_desc(desc);
