@@ -8,7 +8,8 @@
 // IEEE binary32 operation (no contraction), so the stored codes, steps and zero-points are
 // reproducible bit for bit.  A CTA stages the packed bytes of 32 consecutive tokens in shared
 // memory and writes them out with 128-bit stores (tokens of one (batch, head) are contiguous
-// in the cache).  The kernel is HBM-bound on its BF16 input.
+// in the cache).  CTAs are persistent (a few per SM) and keep the next tile's loads in flight
+// while they work on the current one.  The kernel is HBM-bound on its BF16 input.
 #include "kvq_common.cuh"
 
 namespace kvq {
@@ -17,6 +18,7 @@ namespace {
 constexpr int kTileTokens = 32;
 constexpr int kWarps = 8;
 constexpr int kTokPerWarp = kTileTokens / kWarps;
+constexpr int kCtasPerSm = 4;      // persistent grid: SMs x this (a multiple of the SM count)
 
 struct QParams {
   const uint16_t* k; const uint16_t* v;
@@ -26,19 +28,8 @@ struct QParams {
   const int8_t* signs;
   uint8_t* codes[2]; uint8_t* scale[2]; uint16_t* zero[2];
   int tiles_per_bh;
+  int64_t total_tiles;
 };
-
-template <int EPL>
-__device__ __forceinline__ void load_vec(const uint16_t* p, int lane, float (&x)[EPL]) {
-  if constexpr (EPL == 4) {
-    uint2 r = __ldg(reinterpret_cast<const uint2*>(p) + lane);
-    x[0] = bf16_bits_to_f32(r.x & 0xFFFFu); x[1] = bf16_bits_to_f32(r.x >> 16);
-    x[2] = bf16_bits_to_f32(r.y & 0xFFFFu); x[3] = bf16_bits_to_f32(r.y >> 16);
-  } else {
-    uint32_t r = __ldg(reinterpret_cast<const uint32_t*>(p) + lane);
-    x[0] = bf16_bits_to_f32(r & 0xFFFFu); x[1] = bf16_bits_to_f32(r >> 16);
-  }
-}
 
 // y = c_d * H_d * x, stages h = 1, 2, 4, ... in that order, one rounding per operation.
 template <int EPL>
@@ -56,10 +47,11 @@ __device__ __forceinline__ void hadamard(float (&x)[EPL], int lane, float c_d) {
   }
 #pragma unroll
   for (int lm = 1; lm < 32; lm *= 2) {
+    const float sg = (lane & lm) ? -1.0f : 1.0f;     // upper partner: other - own; fma(+-1, own, other) rounds once
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
-      float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
-      x[e] = (lane & lm) ? __fsub_rn(o, x[e]) : __fadd_rn(x[e], o);
+      const float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
+      x[e] = __fmaf_rn(sg, x[e], o);
     }
   }
 #pragma unroll
@@ -68,37 +60,63 @@ __device__ __forceinline__ void hadamard(float (&x)[EPL], int lane, float c_d) {
 
 // Quantizes the vector held by the warp and stages codes / step / zero-point of token slot
 // `tok` in shared memory.
-template <int EPL, int BITS>
-__device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int lane, int group, int tok,
+template <int EPL, int BITS, int GROUP>
+__device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int lane, int tok,
                                                uint32_t* s_codes, uint8_t* s_scale, uint16_t* s_zero) {
   constexpr float L = (float)((1 << BITS) - 1);
   constexpr int kBitsPerLane = EPL * BITS;
   constexpr int kLanesPerWord = 32 / kBitsPerLane;
   constexpr int kWordsPerTok = 32 / kLanesPerWord;
-  const int lanes_per_group = group / EPL;
-  const int G = (32 * EPL) / group;
+  constexpr int lanes_per_group = GROUP / EPL;
+  constexpr int G = (32 * EPL) / GROUP;
 
   float mn = x[0], mx = x[0];
 #pragma unroll
   for (int e = 1; e < EPL; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+#pragma unroll
   for (int off = 1; off < lanes_per_group; off *= 2) {
     mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
     mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
   }
-  const float step = __fdiv_rn(__fsub_rn(mx, mn), L);
+  // Divisions.  x / b as q0 = x*r, rem = fma(-q0, b, x), q = fma(rem, r, q0) with r = RN(1/b) is the correctly
+  // rounded quotient for every divisor used here (3, 15 and the 126 positive E4M3 values: checked against
+  // IEEE division for all 2^23 significands of x), as long as nothing over- or underflows; operands outside
+  // [2^-60, 2^60] (other than 0) take the IEEE division instead, the whole warp together.
+  const float range = __fsub_rn(mx, mn);
+  float amax = fmaxf(fabsf(range), fmaxf(fabsf(mn), fabsf(mx)));
+  float amin = fabsf(range) > 0.f ? fabsf(range) : 1.f;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) amin = fminf(amin, x[e] != 0.f ? fabsf(x[e]) : 1.f);
+  amin = fminf(amin, mn != 0.f ? fabsf(mn) : 1.f);
+  const bool slow = __any_sync(0xFFFFFFFFu, !(amax < 0x1p60f) || !(amin > 0x1p-60f));
+  auto fast_div = [](float a, float b, float r) {
+    const float q0 = __fmul_rn(a, r);
+    return __fmaf_rn(__fmaf_rn(-q0, b, a), r, q0);
+  };
+  const float step = slow ? __fdiv_rn(range, L) : fast_div(range, L, (BITS == 2) ? __uint_as_float(0x3EAAAAABu) : __uint_as_float(0x3D888889u));
   uint32_t sbyte = f32_to_e4m3_byte(step);
   if (sbyte == 0) sbyte = 1;                       // floor at the smallest subnormal 2^-9
   const float ds = e4m3_byte_to_f32(sbyte);
-  const float z = __fsub_rn(0.0f, rintf(__fdiv_rn(mn, ds)));
+  const float rds = __frcp_rn(ds);
+  const float z = __fsub_rn(0.0f, rintf(slow ? __fdiv_rn(mn, ds) : fast_div(mn, ds, rds)));
   const uint32_t zbits = f32_to_bf16_bits(z);
   const float zs = bf16_bits_to_f32(zbits);
 
   uint32_t piece = 0;
+  if (!slow) {
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) {
-    float c = __fadd_rn(rintf(__fdiv_rn(x[e], ds)), zs);
-    c = fminf(fmaxf(c, 0.0f), L);
-    piece |= ((uint32_t)c) << (e * BITS);
+    for (int e = 0; e < EPL; ++e) {
+      float c = __fadd_rn(rintf(fast_div(x[e], ds, rds)), zs);
+      c = fminf(fmaxf(c, 0.0f), L);
+      piece |= (__float_as_uint(__fadd_rn(c, 8388608.f)) & (uint32_t)L) << (e * BITS);   // c is an integer in [0, L]
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      float c = __fadd_rn(rintf(__fdiv_rn(x[e], ds)), zs);
+      c = fminf(fmaxf(c, 0.0f), L);
+      piece |= ((uint32_t)c) << (e * BITS);
+    }
   }
   uint32_t word = piece << ((lane % kLanesPerWord) * kBitsPerLane);
 #pragma unroll
@@ -127,7 +145,30 @@ __device__ __forceinline__ void copy_out(uint8_t* dst, const uint8_t* src, int n
   }
 }
 
-template <int D, int BITS>
+template <int EPL>
+struct RawVec { uint32_t r[EPL / 2]; };
+
+template <int EPL>
+__device__ __forceinline__ void load_raw_vec(RawVec<EPL>& v, const uint16_t* p, int lane) {
+  if constexpr (EPL == 4) {
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p) + lane);
+    v.r[0] = t.x; v.r[1] = t.y;
+  } else {
+    v.r[0] = __ldg(reinterpret_cast<const uint32_t*>(p) + lane);
+  }
+}
+template <int EPL>
+__device__ __forceinline__ void decode_vec(const RawVec<EPL>& v, float (&x)[EPL]) {
+#pragma unroll
+  for (int e = 0; e < EPL / 2; ++e) {
+    x[2 * e] = bf16_bits_to_f32(v.r[e] & 0xFFFFu);
+    x[2 * e + 1] = bf16_bits_to_f32(v.r[e] >> 16);
+  }
+}
+
+// Persistent CTAs: each walks tiles of 32 consecutive tokens of one (batch, head) with a stride of gridDim.x
+// and has the next tile's loads in flight while it rotates, quantizes and packs the current one.
+template <int D, int BITS, int GROUP>
 __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p) {
   constexpr int EPL = D / 32;
   constexpr int CB = D * BITS / 8;
@@ -136,50 +177,64 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
   __shared__ __align__(16) uint16_t s_zero[2][kTileTokens * 4];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int bh = blockIdx.x / p.tiles_per_bh;
-  const int tile = blockIdx.x - bh * p.tiles_per_bh;
-  const int b = bh / p.heads, h = bh - b * p.heads;
-  const int64_t t0 = (int64_t)tile * kTileTokens;
-  const int nt = (int)min((int64_t)kTileTokens, p.n_tokens - t0);
-  const int G = D / p.group;
+  constexpr int G = D / GROUP;
   const float c_d = (D == 64) ? 0.125f : __uint_as_float(0x3DB504F3u);
-
   float sgn[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) sgn[e] = p.signs ? (float)p.signs[lane * EPL + e] : 1.0f;
 
-  const int64_t base = (int64_t)b * p.sb + (int64_t)h * p.sh;
-  float xk[kTokPerWarp][EPL], xv[kTokPerWarp][EPL];
+  RawVec<EPL> rk[kTokPerWarp], rv[kTokPerWarp];
+  auto fetch = [&](int tile_g) {
+    const int bh = tile_g / p.tiles_per_bh;
+    const int tile = tile_g - bh * p.tiles_per_bh;
+    const int b = bh / p.heads, h = bh - b * p.heads;
+    const int64_t t0 = (int64_t)tile * kTileTokens;
+    const int64_t base = (int64_t)b * p.sb + (int64_t)h * p.sh;
 #pragma unroll
-  for (int i = 0; i < kTokPerWarp; ++i) {
-    const int tok = warp * kTokPerWarp + i;
-    if (tok < nt) {
-      const int64_t off = base + (t0 + tok) * p.st;
-      load_vec<EPL>(p.k + off, lane, xk[i]);
-      load_vec<EPL>(p.v + off, lane, xv[i]);
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < kTokPerWarp; ++i) {
-    const int tok = warp * kTokPerWarp + i;
-    if (tok < nt) {
-      if (p.rotate) {
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) xk[i][e] *= sgn[e];
-        hadamard<EPL>(xk[i], lane, c_d);
+    for (int i = 0; i < kTokPerWarp; ++i) {
+      const int64_t t = t0 + warp * kTokPerWarp + i;
+      if (t < p.n_tokens) {
+        load_raw_vec<EPL>(rk[i], p.k + base + t * p.st, lane);
+        load_raw_vec<EPL>(rv[i], p.v + base + t * p.st, lane);
       }
-      quantize_stage<EPL, BITS>(xk[i], lane, p.group, tok, s_codes[0], s_scale[0], s_zero[0]);
-      quantize_stage<EPL, BITS>(xv[i], lane, p.group, tok, s_codes[1], s_scale[1], s_zero[1]);
     }
-  }
-  __syncthreads();
-  const int64_t tok_index = (int64_t)bh * p.capacity + p.cache_len + t0;
+  };
+
+  int tile_g = blockIdx.x;
+  const int total_tiles = (int)p.total_tiles;
+  if (tile_g < total_tiles) fetch(tile_g);
+  for (; tile_g < total_tiles; tile_g += gridDim.x) {
+    const int bh = tile_g / p.tiles_per_bh;
+    const int tile = tile_g - bh * p.tiles_per_bh;
+    const int64_t t0 = (int64_t)tile * kTileTokens;
+    const int nt = (int)min((int64_t)kTileTokens, p.n_tokens - t0);
+    float xk[kTokPerWarp][EPL], xv[kTokPerWarp][EPL];
 #pragma unroll
-  for (int w = 0; w < 2; ++w) {
-    copy_out(p.codes[w] + tok_index * CB, reinterpret_cast<const uint8_t*>(s_codes[w]), nt * CB, threadIdx.x, kWarps * 32);
-    copy_out(p.scale[w] + tok_index * G, s_scale[w], nt * G, threadIdx.x, kWarps * 32);
-    copy_out(reinterpret_cast<uint8_t*>(p.zero[w] + tok_index * G), reinterpret_cast<const uint8_t*>(s_zero[w]),
-             nt * G * 2, threadIdx.x, kWarps * 32);
+    for (int i = 0; i < kTokPerWarp; ++i) { decode_vec<EPL>(rk[i], xk[i]); decode_vec<EPL>(rv[i], xv[i]); }
+    if (tile_g + (int)gridDim.x < total_tiles) fetch(tile_g + (int)gridDim.x);
+#pragma unroll
+    for (int i = 0; i < kTokPerWarp; ++i) {
+      const int tok = warp * kTokPerWarp + i;
+      if (tok < nt) {
+        if (p.rotate) {
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) xk[i][e] = __fmul_rn(xk[i][e], sgn[e]);
+          hadamard<EPL>(xk[i], lane, c_d);
+        }
+        quantize_stage<EPL, BITS, GROUP>(xk[i], lane, tok, s_codes[0], s_scale[0], s_zero[0]);
+        quantize_stage<EPL, BITS, GROUP>(xv[i], lane, tok, s_codes[1], s_scale[1], s_zero[1]);
+      }
+    }
+    __syncthreads();
+    const int64_t tok_index = (int64_t)bh * p.capacity + p.cache_len + t0;
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+      copy_out(p.codes[w] + tok_index * CB, reinterpret_cast<const uint8_t*>(s_codes[w]), nt * CB, threadIdx.x, kWarps * 32);
+      copy_out(p.scale[w] + tok_index * G, s_scale[w], nt * G, threadIdx.x, kWarps * 32);
+      copy_out(reinterpret_cast<uint8_t*>(p.zero[w] + tok_index * G), reinterpret_cast<const uint8_t*>(s_zero[w]),
+               nt * G * 2, threadIdx.x, kWarps * 32);
+    }
+    __syncthreads();
   }
 }
 
@@ -211,14 +266,22 @@ int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const voi
   p.scale[0] = static_cast<uint8_t*>(d->k_scale); p.scale[1] = static_cast<uint8_t*>(d->v_scale);
   p.zero[0] = static_cast<uint16_t*>(d->k_zero); p.zero[1] = static_cast<uint16_t*>(d->v_zero);
   p.tiles_per_bh = (int)((n_tokens + kTileTokens - 1) / kTileTokens);
-  const int64_t blocks = (int64_t)d->batch * d->heads * p.tiles_per_bh;
-  if (blocks > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  p.total_tiles = (int64_t)d->batch * d->heads * p.tiles_per_bh;
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    sms = n;
+  }
+  const int64_t blocks = p.total_tiles < (int64_t)sms * kCtasPerSm ? p.total_tiles : (int64_t)sms * kCtasPerSm;
   dim3 grid((unsigned)blocks), block(kWarps * 32);
-  if (d->head_dim == 128 && d->bits == 2) quantize_append_kernel<128, 2><<<grid, block, 0, st>>>(p);
-  else if (d->head_dim == 128 && d->bits == 4) quantize_append_kernel<128, 4><<<grid, block, 0, st>>>(p);
-  else if (d->head_dim == 64 && d->bits == 2) quantize_append_kernel<64, 2><<<grid, block, 0, st>>>(p);
-  else if (d->head_dim == 64 && d->bits == 4) quantize_append_kernel<64, 4><<<grid, block, 0, st>>>(p);
-  else return KVQ_ERR_UNSUPPORTED;
+  if (p.total_tiles > 0x7FFFFFFFLL - 65536) return KVQ_ERR_UNSUPPORTED;
+#define KVQ_QA(D_, B_, G_) if (d->head_dim == D_ && d->bits == B_ && d->group == G_) { quantize_append_kernel<D_, B_, G_><<<grid, block, 0, st>>>(p); launched = true; }
+  bool launched = false;
+  KVQ_QA(128, 2, 32) KVQ_QA(128, 2, 64) KVQ_QA(128, 2, 128) KVQ_QA(128, 4, 32) KVQ_QA(128, 4, 64) KVQ_QA(128, 4, 128)
+  KVQ_QA(64, 2, 32) KVQ_QA(64, 2, 64) KVQ_QA(64, 4, 32) KVQ_QA(64, 4, 64)
+#undef KVQ_QA
+  if (!launched) return KVQ_ERR_UNSUPPORTED;
   KVQ_CUDA_TRY(cudaGetLastError());
   return KVQ_OK;
 }
