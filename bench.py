@@ -189,7 +189,8 @@ def main():
     peaks = load_peaks()
 
     # ---- set-up (untimed): inputs resident in HBM, cache built chunk by chunk by the append kernel ----
-    wr = inputs.with_seed(w, w.seed + 1000 * rank)
+    from paper_2605_26266_b200 import replicas
+    wr = replicas.replica_workload(w, rank)
 
     def to_dev(bits):
         return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
@@ -256,7 +257,6 @@ def main():
     attn_off_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in recs_off])) if recs_off else float("nan")
 
     # ---- end to end through the public call with HOST buffers ----
-    e2e = None
     if not args.no_e2e:
         hq, hk, hv = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory() for a in (qh, kh, vh))
         hout = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
@@ -278,15 +278,12 @@ def main():
         barrier()
         e2e_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in e2e_recs]))
     # ---- reduce over ranks: slowest rank's time ----
-    t = torch.tensor([step_ms, float(attn_ms.mean()), float(app_ms.mean()), attn_off_ms,
-                      e2e_ms if e2e is None and not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    step_ms, attn_mean, app_mean, attn_off_ms, e2e_ms = [float(x) for x in t.tolist()]
+    step_ms, attn_mean, app_mean, attn_off_ms, e2e_ms = replicas.max_over_ranks(
+        [step_ms, float(attn_ms.mean()), float(app_ms.mean()), attn_off_ms, 0.0 if args.no_e2e else e2e_ms], device=dev)
 
     if rank == 0:
         flops = w.flops()
-        value = world * flops / (step_ms * 1e-3) / 1e12
+        value = replicas.aggregate_value(flops, world, step_ms)
         attn_tf = flops / (attn_mean * 1e-3) / 1e12
         bursty = attn_mean < 1.0
         peak = peaks["tf_burst"] if bursty else peaks["tf_sustained"]
