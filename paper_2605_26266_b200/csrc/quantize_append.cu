@@ -1,15 +1,15 @@
 // Quantize-append kernel: Hadamard rotation (keys), group-wise asymmetric round-to-nearest
 // quantization (Eq. (1)), bit packing and coalesced append of one finished chunk's K and V.
 //
-// One warp owns one token-head vector at a time: lane l holds channels [l*EPL, (l+1)*EPL)
-// (EPL = head_dim/32).  The Walsh-Hadamard butterfly runs its first log2(EPL) stages inside a
-// lane and the remaining five across lanes with shuffles; group minimum/maximum are shuffle
-// reductions over the lanes of a group.  Every add, subtract, multiply and divide is a single
-// IEEE binary32 operation (no contraction), so the stored codes, steps and zero-points are
-// reproducible bit for bit.  A CTA stages the packed bytes of 32 consecutive tokens in shared
-// memory and writes them out with 128-bit stores (tokens of one (batch, head) are contiguous
-// in the cache).  CTAs are persistent (a few per SM) and keep the next tile's loads in flight
-// while they work on the current one.  The kernel is HBM-bound on its BF16 input.
+// Eight lanes own one token-head vector (lane l8 holds channels [l8*EPL, (l8+1)*EPL), EPL = head_dim/8), so a
+// warp works on four vectors at a time.  The Walsh-Hadamard butterfly runs its first log2(EPL) stages inside a
+// lane and the remaining three across lanes with shuffles; group minimum/maximum are shuffle reductions over
+// the lanes of a group, and a lane's codes fill whole 32-bit words.  Every add, subtract, multiply and divide
+// is a single IEEE binary32 operation (no contraction), so the stored codes, steps and zero-points are
+// reproducible bit for bit.  A CTA stages the packed bytes of 32 consecutive tokens in shared memory and
+// writes them out with 128-bit stores (tokens of one (batch, head) are contiguous in the cache).  CTAs are
+// persistent (a few per SM) and keep the next tile's loads in flight while they work on the current one.
+// By its bytes the kernel is HBM-bound on its BF16 input.
 #include "kvq_common.cuh"
 
 namespace kvq {
@@ -18,7 +18,7 @@ namespace {
 constexpr int kTileTokens = 32;
 constexpr int kWarps = 8;
 constexpr int kTokPerWarp = kTileTokens / kWarps;
-constexpr int kCtasPerSm = 4;      // persistent grid: SMs x this (a multiple of the SM count)
+constexpr int kCtasPerSm = 3;      // persistent grid: SMs x this (a multiple of the SM count)
 
 struct QParams {
   const uint16_t* k; const uint16_t* v;
@@ -31,23 +31,25 @@ struct QParams {
   int64_t total_tiles;
 };
 
-// y = c_d * H_d * x, stages h = 1, 2, 4, ... in that order, one rounding per operation.
+// y = c_d * H_d * x for a vector spread over 8 lanes (lane l8 holds channels [l8*EPL, (l8+1)*EPL)):
+// stages h = 1, 2, 4, ... in that order, one rounding per operation.  The first log2(EPL) stages stay in
+// registers, the last three exchange with lanes l8^1, l8^2, l8^4.
 template <int EPL>
-__device__ __forceinline__ void hadamard(float (&x)[EPL], int lane, float c_d) {
+__device__ __forceinline__ void hadamard(float (&x)[EPL], int l8, float c_d) {
 #pragma unroll
   for (int h = 1; h < EPL; h *= 2) {
 #pragma unroll
     for (int i = 0; i < EPL; ++i) {
       if ((i & h) == 0) {
-        float a = x[i], b = x[i + h];
+        const float a = x[i], b = x[i + h];
         x[i] = __fadd_rn(a, b);
         x[i + h] = __fsub_rn(a, b);
       }
     }
   }
 #pragma unroll
-  for (int lm = 1; lm < 32; lm *= 2) {
-    const float sg = (lane & lm) ? -1.0f : 1.0f;     // upper partner: other - own; fma(+-1, own, other) rounds once
+  for (int lm = 1; lm < 8; lm *= 2) {
+    const float sg = (l8 & lm) ? -1.0f : 1.0f;       // upper partner: other - own; fma(+-1, own, other) rounds once
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
       const float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
@@ -58,17 +60,16 @@ __device__ __forceinline__ void hadamard(float (&x)[EPL], int lane, float c_d) {
   for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], c_d);
 }
 
-// Quantizes the vector held by the warp and stages codes / step / zero-point of token slot
-// `tok` in shared memory.
+// Quantizes the vector held by 8 lanes and stages codes / step / zero-point of token slot `tok` in shared
+// memory.  The per-group work (range, step, zero-point) is shared by the GROUP/EPL lanes of a group.
 template <int EPL, int BITS, int GROUP>
-__device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int lane, int tok,
+__device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int l8, int tok,
                                                uint32_t* s_codes, uint8_t* s_scale, uint16_t* s_zero) {
   constexpr float L = (float)((1 << BITS) - 1);
-  constexpr int kBitsPerLane = EPL * BITS;
-  constexpr int kLanesPerWord = 32 / kBitsPerLane;
-  constexpr int kWordsPerTok = 32 / kLanesPerWord;
+  constexpr int kBitsPerLane = EPL * BITS;             // 16, 32 or 64
+  constexpr int kWordsPerTok = 8 * kBitsPerLane / 32;
   constexpr int lanes_per_group = GROUP / EPL;
-  constexpr int G = (32 * EPL) / GROUP;
+  constexpr int G = (8 * EPL) / GROUP;
 
   float mn = x[0], mx = x[0];
 #pragma unroll
@@ -102,29 +103,34 @@ __device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int lane, 
   const uint32_t zbits = f32_to_bf16_bits(z);
   const float zs = bf16_bits_to_f32(zbits);
 
-  uint32_t piece = 0;
+  uint32_t piece[(kBitsPerLane + 31) / 32] = {};
   if (!slow) {
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
       float c = __fadd_rn(rintf(fast_div(x[e], ds, rds)), zs);
       c = fminf(fmaxf(c, 0.0f), L);
-      piece |= (__float_as_uint(__fadd_rn(c, 8388608.f)) & (uint32_t)L) << (e * BITS);   // c is an integer in [0, L]
+      // c is an integer in [0, L]: adding 2^23 leaves it in the low mantissa bits
+      piece[(e * BITS) / 32] |= (__float_as_uint(__fadd_rn(c, 8388608.f)) & (uint32_t)L) << ((e * BITS) % 32);
     }
   } else {
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
       float c = __fadd_rn(rintf(__fdiv_rn(x[e], ds)), zs);
       c = fminf(fmaxf(c, 0.0f), L);
-      piece |= ((uint32_t)c) << (e * BITS);
+      piece[(e * BITS) / 32] |= ((uint32_t)c) << ((e * BITS) % 32);
     }
   }
-  uint32_t word = piece << ((lane % kLanesPerWord) * kBitsPerLane);
-#pragma unroll
-  for (int off = 1; off < kLanesPerWord; off *= 2) word |= __shfl_xor_sync(0xFFFFFFFFu, word, off);
-  if ((lane % kLanesPerWord) == 0) s_codes[tok * kWordsPerTok + lane / kLanesPerWord] = word;
-  if ((lane % lanes_per_group) == 0) {
-    s_scale[tok * G + lane / lanes_per_group] = (uint8_t)sbyte;
-    s_zero[tok * G + lane / lanes_per_group] = (uint16_t)zbits;
+  if constexpr (kBitsPerLane == 16) {                  // two lanes share a word
+    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, piece[0], 1);
+    if ((l8 & 1) == 0) s_codes[tok * kWordsPerTok + (l8 >> 1)] = piece[0] | (other << 16);
+  } else if constexpr (kBitsPerLane == 32) {
+    s_codes[tok * kWordsPerTok + l8] = piece[0];
+  } else {
+    *reinterpret_cast<uint2*>(&s_codes[tok * kWordsPerTok + 2 * l8]) = make_uint2(piece[0], piece[1]);
+  }
+  if ((l8 % lanes_per_group) == 0) {
+    s_scale[tok * G + l8 / lanes_per_group] = (uint8_t)sbyte;
+    s_zero[tok * G + l8 / lanes_per_group] = (uint16_t)zbits;
   }
 }
 
@@ -146,57 +152,56 @@ __device__ __forceinline__ void copy_out(uint8_t* dst, const uint8_t* src, int n
 }
 
 template <int EPL>
-struct RawVec { uint32_t r[EPL / 2]; };
+struct RawVec { uint4 r[EPL / 8]; };      // EPL BF16 values of one lane
 
 template <int EPL>
-__device__ __forceinline__ void load_raw_vec(RawVec<EPL>& v, const uint16_t* p, int lane) {
-  if constexpr (EPL == 4) {
-    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p) + lane);
-    v.r[0] = t.x; v.r[1] = t.y;
-  } else {
-    v.r[0] = __ldg(reinterpret_cast<const uint32_t*>(p) + lane);
-  }
+__device__ __forceinline__ void load_raw_vec(RawVec<EPL>& v, const uint16_t* p, int l8) {
+#pragma unroll
+  for (int i = 0; i < EPL / 8; ++i) v.r[i] = __ldg(reinterpret_cast<const uint4*>(p) + l8 * (EPL / 8) + i);
 }
 template <int EPL>
 __device__ __forceinline__ void decode_vec(const RawVec<EPL>& v, float (&x)[EPL]) {
 #pragma unroll
-  for (int e = 0; e < EPL / 2; ++e) {
-    x[2 * e] = bf16_bits_to_f32(v.r[e] & 0xFFFFu);
-    x[2 * e + 1] = bf16_bits_to_f32(v.r[e] >> 16);
+  for (int i = 0; i < EPL / 8; ++i) {
+    const uint32_t w[4] = {v.r[i].x, v.r[i].y, v.r[i].z, v.r[i].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      x[8 * i + 2 * e] = bf16_bits_to_f32(w[e] & 0xFFFFu);
+      x[8 * i + 2 * e + 1] = bf16_bits_to_f32(w[e] >> 16);
+    }
   }
 }
 
 // Persistent CTAs: each walks tiles of 32 consecutive tokens of one (batch, head) with a stride of gridDim.x
-// and has the next tile's loads in flight while it rotates, quantizes and packs the current one.
+// and has the next tile's loads in flight while it rotates, quantizes and packs the current one.  A warp
+// works on four token-head vectors at a time, eight lanes per vector.
 template <int D, int BITS, int GROUP>
 __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p) {
-  constexpr int EPL = D / 32;
+  constexpr int EPL = D / 8;
   constexpr int CB = D * BITS / 8;
   __shared__ __align__(16) uint32_t s_codes[2][kTileTokens * CB / 4];
   __shared__ __align__(16) uint8_t s_scale[2][kTileTokens * 4];
   __shared__ __align__(16) uint16_t s_zero[2][kTileTokens * 4];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int l8 = lane & 7;
+  const int tok = warp * kTokPerWarp + (lane >> 3);          // token slot inside the tile
   constexpr int G = D / GROUP;
   const float c_d = (D == 64) ? 0.125f : __uint_as_float(0x3DB504F3u);
-  float sgn[EPL];
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) sgn[e] = p.signs ? (float)p.signs[lane * EPL + e] : 1.0f;
 
-  RawVec<EPL> rk[kTokPerWarp], rv[kTokPerWarp];
+  RawVec<EPL> rk, rv;
   auto fetch = [&](int tile_g) {
     const int bh = tile_g / p.tiles_per_bh;
     const int tile = tile_g - bh * p.tiles_per_bh;
     const int b = bh / p.heads, h = bh - b * p.heads;
-    const int64_t t0 = (int64_t)tile * kTileTokens;
-    const int64_t base = (int64_t)b * p.sb + (int64_t)h * p.sh;
+    const int64_t t = (int64_t)tile * kTileTokens + tok;
+    if (t < p.n_tokens) {
+      const int64_t off = (int64_t)b * p.sb + (int64_t)h * p.sh + t * p.st;
+      load_raw_vec<EPL>(rk, p.k + off, l8);
+      load_raw_vec<EPL>(rv, p.v + off, l8);
+    } else {                                                  // slots past the end quantize zeros, never stored
 #pragma unroll
-    for (int i = 0; i < kTokPerWarp; ++i) {
-      const int64_t t = t0 + warp * kTokPerWarp + i;
-      if (t < p.n_tokens) {
-        load_raw_vec<EPL>(rk[i], p.k + base + t * p.st, lane);
-        load_raw_vec<EPL>(rv[i], p.v + base + t * p.st, lane);
-      }
+      for (int i = 0; i < EPL / 8; ++i) { rk.r[i] = make_uint4(0, 0, 0, 0); rv.r[i] = make_uint4(0, 0, 0, 0); }
     }
   };
 
@@ -208,23 +213,20 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
     const int tile = tile_g - bh * p.tiles_per_bh;
     const int64_t t0 = (int64_t)tile * kTileTokens;
     const int nt = (int)min((int64_t)kTileTokens, p.n_tokens - t0);
-    float xk[kTokPerWarp][EPL], xv[kTokPerWarp][EPL];
-#pragma unroll
-    for (int i = 0; i < kTokPerWarp; ++i) { decode_vec<EPL>(rk[i], xk[i]); decode_vec<EPL>(rv[i], xv[i]); }
+    float x[EPL];
+    decode_vec<EPL>(rk, x);
+    const RawVec<EPL> rv_cur = rv;
     if (tile_g + (int)gridDim.x < total_tiles) fetch(tile_g + (int)gridDim.x);
+    if (p.rotate) {
+      if (p.signs) {
 #pragma unroll
-    for (int i = 0; i < kTokPerWarp; ++i) {
-      const int tok = warp * kTokPerWarp + i;
-      if (tok < nt) {
-        if (p.rotate) {
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) xk[i][e] = __fmul_rn(xk[i][e], sgn[e]);
-          hadamard<EPL>(xk[i], lane, c_d);
-        }
-        quantize_stage<EPL, BITS, GROUP>(xk[i], lane, tok, s_codes[0], s_scale[0], s_zero[0]);
-        quantize_stage<EPL, BITS, GROUP>(xv[i], lane, tok, s_codes[1], s_scale[1], s_zero[1]);
+        for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], (float)p.signs[l8 * EPL + e]);
       }
+      hadamard<EPL>(x, l8, c_d);
     }
+    quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[0], s_scale[0], s_zero[0]);
+    decode_vec<EPL>(rv_cur, x);
+    quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[1], s_scale[1], s_zero[1]);
     __syncthreads();
     const int64_t tok_index = (int64_t)bh * p.capacity + p.cache_len + t0;
 #pragma unroll
