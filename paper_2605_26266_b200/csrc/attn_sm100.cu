@@ -68,8 +68,8 @@ enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull 
            kODone = 13, kQCurDone = 15, kQRotFull = 16, kDrain = 17, kQEmpty = 18, kOFree = 19,
            kPair = 21 /* 8: [query tile][lane quarter], the two warps that share 32 rows */ };
 
-constexpr long long kTimeoutCycles = 2000000000LL;   // about a second
-constexpr long long kDrainCycles = 20000000LL;
+constexpr uint32_t kTimeoutCycles = 2000000000u;   // about a second; 32-bit clock differences stay exact below 2^32
+constexpr uint32_t kDrainCycles = 20000000u;
 constexpr float kLog2e = 1.4426950408889634f;
 // registers per thread after reallocation: 128 * 72 + 256 * 168 + 128 * 96 = 64512 <= 65536
 constexpr int kRegsIssue = 72, kRegsSoftmax = 168, kRegsDequant = 96;
@@ -88,30 +88,46 @@ struct TParams {
   float ax_coef;           // -sigma / 24
   float* lse; float* cached_mass;
   int32_t* status;
-  // persistent schedule: units = (batch*head, 256-row query block); every unit has `tiles` key tiles;
-  // the n_units * tiles tile steps are cut into gridDim.x equal contiguous ranges
+  // schedule: units = (batch*head, 256-row query block); every unit has `tiles` key tiles (see Schedule)
   int q_blocks, n_units, tiles;
+  int n_whole;             // units [0, n_whole) are computed whole; the rest are split over all CTAs
   float* partial;          // workspace: 2 slots per CTA, see kSlotFloats
 };
 
 // One partial result: unnormalised O [256][128] FP32, then m[256], l_cur[256], l_cached[256]
 constexpr int kSlotFloats = 256 * kD + 3 * 256;
 
-// A contiguous run of key tiles [tb, te) of one unit.
-struct Segment { int unit, tb, te; };
+// A contiguous run of key tiles [tb, te) of one unit; `slot` is the CTA's partial-result slot if the run is
+// not the whole unit.
+struct Segment { int unit, tb, te, slot; };
+// Work of one CTA.  Units [0, n_whole) are computed whole, CTA c taking units c, c + n_ctas, ... so that
+// neighbouring CTAs walk the key tiles of neighbouring units (mostly the same head) at the same time and
+// share them in L2.  The key-tile steps of the remaining units are cut into n_ctas equal contiguous
+// ranges, one per CTA.  n_units * tiles < 2^31 (checked on the host).
 struct Schedule {
-  int g, g_end, tiles;     // n_units * tiles < 2^31 (checked on the host)
-  __device__ __forceinline__ Schedule(int cta, int n_ctas, int n_units, int tiles_) : tiles(tiles_) {
-    const long long W = (long long)n_units * tiles_;
-    g = (int)(W * cta / n_ctas);
-    g_end = (int)(W * (cta + 1) / n_ctas);
+  int tiles, n_ctas, n_whole;
+  int u;                   // next whole unit of this CTA
+  int g, g_end, first;     // range in the split part (tile steps counted from unit n_whole); its first unit
+  __device__ __forceinline__ Schedule(int cta, int n_ctas_, const TParams& p)
+      : tiles(p.tiles), n_ctas(n_ctas_), n_whole(p.n_whole), u(cta) {
+    const long long Wr = (long long)(p.n_units - p.n_whole) * p.tiles;
+    g = (int)(Wr * cta / n_ctas_);
+    g_end = (int)(Wr * (cta + 1) / n_ctas_);
+    first = n_whole + g / max(tiles, 1);
   }
   __device__ __forceinline__ bool next(Segment& sg) {
+    if (u < n_whole) {
+      sg.unit = u; sg.tb = 0; sg.te = tiles; sg.slot = 0;
+      u += n_ctas;
+      return true;
+    }
     if (g >= g_end) return false;
-    sg.unit = g / tiles;
-    sg.tb = g - sg.unit * tiles;
+    const int ru = g / tiles;
+    sg.unit = n_whole + ru;
+    sg.tb = g - ru * tiles;
     const int n = min(tiles - sg.tb, g_end - g);
     sg.te = sg.tb + n;
+    sg.slot = sg.unit == first ? 0 : 1;
     g += n;
     return true;
   }
@@ -119,29 +135,25 @@ struct Schedule {
 
 struct Ctx {
   uint32_t bar0;
-  volatile int* abort;
-  int32_t* status;
+  volatile int* abort;     // shared-memory word: 0, or the diagnostic code of the wait that gave up
   __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * i; }
-  // Bounded wait; false once the CTA is aborting.
+  // Bounded wait; false once the CTA is aborting.  Written to be small: it is inlined at some forty
+  // sites, and the roles' loops have to stay resident in the SM's instruction cache.
   __device__ __forceinline__ bool wait(int i, uint32_t parity, int code) const {
     const uint32_t b = bar(i);
     if (mbar_try_wait(b, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-      if (mbar_try_wait(b, parity)) return true;
+    const uint32_t t0 = (uint32_t)clock();
+    while (!mbar_try_wait(b, parity)) {
       if (*abort) return false;
-      if (clock64() - t0 > kTimeoutCycles) {
-        *abort = 1;
-        if (status) atomicCAS(status, 0, code);
-        return false;
-      }
+      if ((uint32_t)clock() - t0 > kTimeoutCycles) { *abort = code; return false; }
     }
+    return true;
   }
   // Used only on the way out: lets work already in flight finish, ignoring the abort flag.
   __device__ __forceinline__ void drain(int i, uint32_t parity) const {
     const uint32_t b = bar(i);
-    const long long t0 = clock64();
-    while (!mbar_try_wait(b, parity) && clock64() - t0 < kDrainCycles) {}
+    const uint32_t t0 = (uint32_t)clock();
+    while (!mbar_try_wait(b, parity) && (uint32_t)clock() - t0 < kDrainCycles) {}
   }
 };
 
@@ -429,7 +441,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   volatile int* misc = reinterpret_cast<volatile int*>(smem + kOffMisc);   // [0] tmem base, [1] abort flag
-  Ctx cx{sbase + kOffBar, misc + 1, p.status};
+  Ctx cx{sbase + kOffBar, misc + 1};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_rt = (p.n_cur + kBlockN - 1) / kBlockN;
@@ -478,7 +490,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
-      Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+      Schedule sch(blockIdx.x, gridDim.x, p);
       Segment sg;
       int it = 0, nseg = 0, issued_it = -1;
       bool ok = true;
@@ -574,7 +586,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         __syncwarp();
       };
-      Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+      Schedule sch(blockIdx.x, gridDim.x, p);
       Segment sg;
       int it = 0, nseg = 0;
       bool ok = true;
@@ -583,54 +595,48 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // last current-chunk tile of this segment (-1 if the segment starts in the cache): after its
         // score MMAs nothing reads the unrotated query any more
         const int t_lastcur = (sg.tb < n_rt) ? min(sg.te, n_rt) - 1 : -1;
+        const int t_rot = max(sg.tb, n_rt);          // first cached tile: its scores need the rotated query
         if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, sp, 201)))) break;
-        {
-          const bool cached0 = sg.tb >= n_rt;
-          if (cached0) {
-            commit1(cx.bar(kQCurDone));
-            if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQRotFull, sp, 207)))) break;
-          }
-          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + (it & 1), (it >> 1) & 1, 202)))) break;
-          tc_fence_after();
-          issue_qk(0, it & 1, cached0);
-          issue_qk(1, it & 1, cached0);
-          commit1(cx.bar(kKEmpty + (it & 1)));
-          if (sg.tb == t_lastcur) commit1(cx.bar(kQCurDone));
-        }
-        for (int t = sg.tb; t < sg.te; ++t, ++it) {
-          const int s = it & 1;
-          const uint32_t ph = (it >> 1) & 1;
+        // Iteration t issues O += P V of tile t and S = Q K^T of tile t + 1 (t = tb - 1: only the scores of
+        // the first tile).  The four MMA groups of an iteration go through ONE rolled loop, so that the
+        // issue code exists once and the warp's loop stays small in the instruction cache.  Order:
+        // PV0 QK0 PV1 QK1; if tile t + 1 is the first cached one, PV0 PV1 QK0 QK1, because its scores have
+        // to wait for the query rotation, which itself waits for every earlier score MMA.
+        --it;
+        for (int t = sg.tb - 1; ok && t < sg.te; ++t, ++it) {
+          const bool has_pv = t >= sg.tb, has_qk = t + 1 < sg.te;
           const bool first = t == sg.tb;
-          const bool next = t + 1 < sg.te;
-          const bool switch_next = next && (t + 1 == n_rt);
+          const bool rot = has_qk && (t + 1 == t_rot);
           const bool next_cached = t + 1 >= n_rt;
-          const int s1 = (it + 1) & 1;
-          const uint32_t ph1 = ((it + 1) >> 1) & 1;
-          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kVFull + s, ph, 203)))) break;
-          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kPFull + 0, it & 1, 204)))) break;
-          if (first && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kOFree + 0, sp ^ 1, 209)))) break;   // previous segment's O has been read out
-          tc_fence_after();
-          issue_pv(0, s, !first);
-          if (next && !switch_next) {
-            if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + s1, ph1, 205)))) break;
-            tc_fence_after();
-            issue_qk(0, s1, next_cached);
-          }
-          if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kPFull + 1, it & 1, 206)))) break;
-          if (first && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kOFree + 1, sp ^ 1, 210)))) break;
-          tc_fence_after();
-          issue_pv(1, s, !first);
-          commit1(cx.bar(kVEmpty + s));
-          if (next) {
-            if (switch_next) {
-              if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQRotFull, sp, 207)))) break;
-              if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + s1, ph1, 208)))) break;
+          const int s = it & 1, s1 = (it + 1) & 1;
+          const uint32_t ph = (it >> 1) & 1, ph1 = ((it + 1) >> 1) & 1;
+          if (rot && !has_pv) commit1(cx.bar(kQCurDone));        // the segment starts in the cache
+#pragma unroll 1
+          for (int step = 0; step < 4; ++step) {
+            const int op = rot ? step : (((step & 1) << 1) | (step >> 1));   // bit 1: scores, bit 0: query tile
+            const int qt = op & 1;
+            if (op < 2) {
+              if (!has_pv) continue;
+              if (qt == 0 && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kVFull + s, ph, 203)))) break;
+              if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kPFull + qt, it & 1, 204)))) break;
+              // first tile of a segment: the previous segment's O must have been read out
+              if (first && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kOFree + qt, sp ^ 1, 209)))) break;
               tc_fence_after();
-              issue_qk(0, s1, true);
+              issue_pv(qt, s, !first);
+              if (qt == 1) commit1(cx.bar(kVEmpty + s));
+            } else {
+              if (!has_qk) continue;
+              if (qt == 0) {
+                if (rot && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQRotFull, sp, 207)))) break;
+                if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + s1, ph1, 205)))) break;
+                tc_fence_after();
+              }
+              issue_qk(qt, s1, next_cached);
+              if (qt == 1) {
+                commit1(cx.bar(kKEmpty + s1));
+                if (t + 1 == t_lastcur) commit1(cx.bar(kQCurDone));
+              }
             }
-            issue_qk(1, s1, next_cached);
-            commit1(cx.bar(kKEmpty + s1));
-            if (t + 1 == t_lastcur) commit1(cx.bar(kQCurDone));
           }
         }
         if (!ok) break;
@@ -655,18 +661,21 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const float c_row = p.scale_log2;
     float* xmax = reinterpret_cast<float*>(smem + kOffXmax);
     float* xl = reinterpret_cast<float*>(smem + kOffXl);
-    Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+    Schedule sch(blockIdx.x, gridDim.x, p);
     Segment sg;
     int it = 0, nseg = 0;
     uint32_t pair_phase = 0;                                  // pair barriers flip once per tile and once per epilogue
     bool ok = true;
     while (ok && sch.next(sg)) {
-      float m[2] = {-INFINITY, -INFINITY}, l_cur[2] = {0.f, 0.f}, l_cac[2] = {0.f, 0.f};
+      // Running max and row sums (current / cached keys) of the query tile being worked on (m_a ...) and of
+      // the other one (m_b ...).  The loops over the two query tiles are rolled, to keep this role's code
+      // small in the instruction cache, and swap the two sets at the end of each pass.
+      float m_a = -INFINITY, m_b = -INFINITY, lcur_a = 0.f, lcur_b = 0.f, lcac_a = 0.f, lcac_b = 0.f;
       uint32_t sr[64];                           // this thread's 64 scores, then its 32 packed probabilities
       for (int t = sg.tb; ok && t < sg.te; ++t, ++it) {
         const bool cached = t >= n_rt;
         const int n_valid = (cached ? min(kBlockN, p.n_cached - (t - n_rt) * kBlockN) : min(kBlockN, p.n_cur - t * kBlockN)) - half * 64;
-#pragma unroll
+#pragma unroll 1
         for (int qt = 0; qt < 2; ++qt) {
           const int r256 = qt * kBlockM + r128;
           const uint32_t s_addr = tmem + lane_addr + qt * 128 + half * 64;
@@ -696,13 +705,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           ok = __all_sync(0xFFFFFFFFu, cx.wait(kPair + qt * 4 + wq, pair_phase, 304));
           if (!ok) break;
           tc_fence_after();
-          const float m_new = fmaxf(m[qt], fmaxf(mine, xmax[(half ^ 1) * 256 + r256]) * c_row);
-          if (__any_sync(0xFFFFFFFFu, m_new - m[qt] > kRescaleThreshold)) {
+          const float m_new = fmaxf(m_a, fmaxf(mine, xmax[(half ^ 1) * 256 + r256]) * c_row);
+          if (__any_sync(0xFFFFFFFFu, m_new - m_a > kRescaleThreshold)) {
             if (t > sg.tb) {
               ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (it - 1) & 1, 302));
               if (!ok) break;
               tc_fence_after();
-              const float f = ex2(m[qt] - m_new);
+              const float f = ex2(m_a - m_new);
 #pragma unroll 1
               for (int c = 0; c < 4; ++c) {
                 uint32_t r[16];
@@ -712,11 +721,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
                 tmem_st16(o_addr + 16 * c, r);
               }
-              l_cur[qt] *= f; l_cac[qt] *= f;
+              lcur_a *= f; lcac_a *= f;
             }
-            m[qt] = m_new;
+            m_a = m_new;
           }
-          const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m[qt], -m[qt]);
+          const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m_a, -m_a);
           float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
           for (int i = 0; i < 64; i += 2) {
@@ -727,10 +736,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             sr[i >> 1] = cvt_bf16x2(pr.x, pr.y);
           }
           tmem_st32(p_addr, sr);
-          if (cached) l_cac[qt] += sum2.x + sum2.y; else l_cur[qt] += sum2.x + sum2.y;
+          if (cached) lcac_a += sum2.x + sum2.y; else lcur_a += sum2.x + sum2.y;
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(cx.bar(kPFull + qt));
+          { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
         }
         pair_phase ^= 1;
       }
@@ -738,8 +748,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // ---- segment epilogue: read O out of TMEM, release it, combine the two column halves' row sums ----
       const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
       const bool whole = sg.tb == 0 && sg.te == T;
-      float* slot = p.partial + (size_t)(2 * blockIdx.x + (nseg > 0 ? 1 : 0)) * kSlotFloats;   // partial segments only
-#pragma unroll
+      float* slot = p.partial + (size_t)(2 * blockIdx.x + sg.slot) * kSlotFloats;   // partial segments only
+#pragma unroll 1
       for (int qt = 0; qt < 2; ++qt) {
         const int r256 = qt * kBlockM + r128;
         const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128 + half * 64;
@@ -751,13 +761,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(cx.bar(kOFree + qt));
-        xl[(half * 256 + r256) * 2] = l_cur[qt];
-        xl[(half * 256 + r256) * 2 + 1] = l_cac[qt];
+        xl[(half * 256 + r256) * 2] = lcur_a;
+        xl[(half * 256 + r256) * 2 + 1] = lcac_a;
         mbar_arrive(cx.bar(kPair + qt * 4 + wq));
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kPair + qt * 4 + wq, pair_phase, 305));
         if (!ok) break;
-        const float lc = l_cur[qt] + xl[((half ^ 1) * 256 + r256) * 2];
-        const float la = l_cac[qt] + xl[((half ^ 1) * 256 + r256) * 2 + 1];
+        const float lc = lcur_a + xl[((half ^ 1) * 256 + r256) * 2];
+        const float la = lcac_a + xl[((half ^ 1) * 256 + r256) * 2 + 1];
         const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
         if (whole) {
           if (row < p.m_tokens) {
@@ -775,7 +785,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             if (half == 0) {
               const int64_t idx = (int64_t)bh * p.m_tokens + row;
-              if (p.lse) p.lse[idx] = (m[qt] + log2f(l)) * 0.6931471805599453f;
+              if (p.lse) p.lse[idx] = (m_a + log2f(l)) * 0.6931471805599453f;
               if (p.cached_mass) p.cached_mass[idx] = la * inv;
             }
           }
@@ -785,11 +795,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int i = 0; i < 64; i += 4)
             orow[i >> 2] = make_float4(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1]), __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
           if (half == 0) {
-            slot[256 * kD + r256] = m[qt];
+            slot[256 * kD + r256] = m_a;
             slot[256 * kD + 256 + r256] = lc;
             slot[256 * kD + 512 + r256] = la;
           }
         }
+        { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
       }
       pair_phase ^= 1;
       ++nseg;
@@ -799,7 +810,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // ================= dequant + query rotation =================
     setmaxnreg_dec<kRegsDequant>();
     const int dt = tid - 12 * 32;          // 0..127: the key of the tile this thread expands
-    Schedule sch(blockIdx.x, gridDim.x, p.n_units, T);
+    Schedule sch(blockIdx.x, gridDim.x, p);
     Segment sg;
     int it = 0, nseg = 0;
     bool ok = true;
@@ -859,16 +870,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
+    // a wait that gave up left its diagnostic code in the abort word: report the first one
+    if (lane == 0 && misc[1] != 0 && p.status) atomicCAS(p.status, 0, misc[1]);
   }
 }
 
 // Combines the partial results of every unit whose key tiles were split over several CTAs.
-// grid (n_units, 32): a block handles 8 rows x 128 columns; thread = (row, 8-column group).
+// grid (n_units - n_whole, 32): a block handles 8 rows x 128 columns; thread = (row, 8-column group).
 __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_ctas) {
-  const int unit = blockIdx.x;
+  const int unit = p.n_whole + blockIdx.x;
   const int T = p.tiles;
-  const long long W = (long long)p.n_units * T;
-  const long long g_lo = (long long)unit * T, g_hi = g_lo + T;
+  const long long W = (long long)(p.n_units - p.n_whole) * T;     // tile steps of the split part
+  const long long g_lo = (long long)blockIdx.x * T, g_hi = g_lo + T;
   auto start = [&](long long c) { return W * c / n_ctas; };
   auto owner = [&](long long g) {
     long long c = g * n_ctas / W;
@@ -885,13 +898,13 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_
   if (row >= p.m_tokens) return;
   float m = -INFINITY;
   for (int c = c_first; c <= c_last; ++c) {
-    const int slot = 2 * c + ((int)(start(c) / T) == unit ? 0 : 1);
+    const int slot = 2 * c + (p.n_whole + (int)(start(c) / T) == unit ? 0 : 1);
     m = fmaxf(m, p.partial[(size_t)slot * kSlotFloats + 256 * kD + r256]);
   }
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   float l_cur = 0.f, l_cac = 0.f;
   for (int c = c_first; c <= c_last; ++c) {
-    const int slot = 2 * c + ((int)(start(c) / T) == unit ? 0 : 1);
+    const int slot = 2 * c + (p.n_whole + (int)(start(c) / T) == unit ? 0 : 1);
     const float* sl = p.partial + (size_t)slot * kSlotFloats;
     const float f = exp2f(sl[256 * kD + r256] - m);
     l_cur += f * sl[256 * kD + 256 + r256];
@@ -962,19 +975,28 @@ int num_sms() {
   return cached;
 }
 
-// Grid policy.  With at least half as many units as SMs every CTA takes one whole unit (no partial results,
-// the hardware scheduler balances the waves; measured faster than splitting on the chunk-sized workloads).
-// With fewer units (short query chunk, long cache) the n_units * tiles key-tile steps are cut into equal
-// contiguous ranges, one per SM, each at least ~4 tiles long, and split units are merged afterwards.
-int grid_ctas(int64_t n_units, int64_t tiles) {
+// Grid policy: how many CTAs, and how many leading units are computed whole (the rest are split).
+//  * At least as many units as SMs: one persistent CTA per SM.  Whole units are dealt out in rounds of
+//    one per CTA; the last, incomplete round of R units would leave SMs idle for a whole unit's time, so
+//    when R is at most half the SMs its key-tile steps are split evenly over all CTAs instead.
+//  * Between half as many and as many units as SMs: one CTA per unit, nothing split (splitting measured
+//    slower than the idle SMs cost).
+//  * Fewer (short query chunk, long cache): all tile steps are cut into equal ranges, one per CTA, each at
+//    least ~4 tiles long.
+struct Plan { int ctas; int n_whole; };
+Plan plan_grid(int64_t n_units, int64_t tiles) {
   const int sms = num_sms();
-  if (2 * n_units >= sms) return (int)n_units;
+  if (n_units >= sms) {
+    const int64_t r = n_units % sms;
+    return {sms, (int)((r == 0 || 2 * r > sms) ? n_units : n_units - r)};
+  }
+  if (2 * n_units >= sms) return {(int)n_units, (int)n_units};
   const int64_t W = n_units * tiles;
   int64_t c = W / 4;
   if (c < n_units) c = n_units;
   if (c > sms) c = sms;
   if (c > W) c = W;
-  return (int)(c < 1 ? 1 : c);
+  return {(int)(c < 1 ? 1 : c), 0};
 }
 
 template <int BITS, int GROUP>
@@ -986,8 +1008,8 @@ int launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, 
   }
   attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
   KVQ_CUDA_TRY(cudaGetLastError());
-  if ((int)grid.x != p.n_units) {   // units were split over CTAs: combine their partial results
-    attn_merge_kernel<<<dim3((unsigned)p.n_units, 32), 128, 0, st>>>(p, (int)grid.x);
+  if (p.n_whole != p.n_units) {   // units were split over CTAs: combine their partial results
+    attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 32), 128, 0, st>>>(p, (int)grid.x);
     KVQ_CUDA_TRY(cudaGetLastError());
   }
   return KVQ_OK;
@@ -1010,8 +1032,8 @@ size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, 
   if (m_tokens <= 0) return 0;
   int64_t qb, nu, tiles;
   schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
-  const int c = grid_ctas(nu, tiles);
-  return c != nu ? (size_t)c * 2 * kSlotFloats * sizeof(float) : 0;
+  const Plan pl = plan_grid(nu, tiles);
+  return pl.n_whole != nu ? (size_t)pl.ctas * 2 * kSlotFloats * sizeof(float) : 0;
 }
 
 int launch_attn_tcgen05(const AttnArgs& a) {
@@ -1041,7 +1063,9 @@ int launch_attn_tcgen05(const AttnArgs& a) {
   if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
   p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
   p.partial = static_cast<float*>(a.workspace);
-  dim3 grid((unsigned)grid_ctas(nu, tiles));
+  const Plan pl = plan_grid(nu, tiles);
+  p.n_whole = pl.n_whole;
+  dim3 grid((unsigned)pl.ctas);
   if (d->bits == 2) {
     if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
     if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);
@@ -1086,14 +1110,18 @@ int launch_attn_tcgen05_static(const AttnArgs& a) {
   int64_t qb, nu, tiles;
   schedule_shape(d, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
   if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
-  int ctas = grid_ctas(nu, tiles);
+  Plan pl = plan_grid(nu, tiles);
   float* scratch = nullptr;
-  if (ctas != nu) {                                        // units are split: partial results need the scratch
-    if (nu > kStaticMaxCtas) return KVQ_ERR_WORKSPACE;     // stated maximum: 32 units when splitting
-    if (ctas > kStaticMaxCtas) ctas = kStaticMaxCtas;
-    if (ctas < nu) ctas = (int)nu;
-    const int r = static_scratch_ptr(&scratch);
-    if (r != KVQ_OK) return r;
+  if (pl.n_whole != nu) {
+    if (pl.n_whole > 0) {
+      pl.n_whole = (int)nu;                                // many units: deal all of them out whole, no scratch
+    } else {                                               // few units, all split: partial results need the scratch
+      if (nu > kStaticMaxCtas) return KVQ_ERR_WORKSPACE;   // stated maximum: 32 units when splitting
+      if (pl.ctas > kStaticMaxCtas) pl.ctas = kStaticMaxCtas;
+      if (pl.ctas < nu) pl.ctas = (int)nu;
+      const int r = static_scratch_ptr(&scratch);
+      if (r != KVQ_OK) return r;
+    }
   }
   EncodeTiledFn enc;
   int r = get_encode_fn(&enc);
@@ -1117,7 +1145,8 @@ int launch_attn_tcgen05_static(const AttnArgs& a) {
   p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
   p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
   p.partial = scratch;
-  dim3 grid((unsigned)ctas);
+  p.n_whole = pl.n_whole;
+  dim3 grid((unsigned)pl.ctas);
   if (d->bits == 2) {
     if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
     if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);

@@ -111,6 +111,19 @@ def test_short_chunk_long_cache_is_split_over_ctas(B):
     assert rc == B.KVQ_ERR_WORKSPACE
 
 
+@pytest.mark.parametrize("heads,picked", [(152, [0, 77, 147, 148, 150, 151]), (230, [0, 147, 148, 229])])
+def test_more_units_than_sms(B, heads, picked):
+    """More (head, query block) units than SMs: persistent CTAs take whole units in rounds; a short last round
+    (152 units on 148 SMs) is split over all CTAs and merged, a long one (230 units) is dealt out whole."""
+    w = inputs.Workload("many", 330 + heads, 1, heads, 128, 200, 0, 2, 32, 0, k_outliers=1, k_outlier_scale=5.0)
+    units = [(0, h) for h in picked]
+    g, o, n, sel = _build(B, w, 3, tokens=150, units=units, cap=512)
+    assert n == 450
+    q, _, _ = inputs.make_chunk(w, 7)
+    _, kc, vc = inputs.make_chunk(w, 8, tokens=130)
+    _compare(B, g, o, n, q, kc, vc, T.sigma_of(128), sel, flags_list=[("tcgen05", B.KVQ_KERNEL_TCGEN05)])
+
+
 def test_empty_cache_is_plain_attention(B):
     w = inputs.Workload("empty", 300, 1, 2, 128, 150, 0, 2, 64, 0)
     g = B.Cache(1, 2, 128, 2, 64, 128)
