@@ -116,7 +116,10 @@ int kvq_quantize_append(const kvq_cache_desc* desc, int64_t cache_len,
                         int64_t n_tokens, kvq_stream_t stream);
 
 /*
- * Bytes of device workspace kvq_attn_corrected needs for this problem (may be 0).
+ * Bytes of device workspace kvq_attn_corrected needs for this problem (may be 0).  With the tcgen05 kernel
+ * and a non-empty cache window it holds the rotated query chunk (Section 3.1: q~ = H q in FP16, plus the
+ * per-group squared norms nu of Eq. 15, 272 bytes per query row, written by a pre-pass kernel of the same
+ * call) and, when the key tiles of a unit are split over several CTAs, their partial results.
  * out_bytes is host memory.  Same errors as kvq_attn_corrected's argument checks.
  */
 int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len,
@@ -170,20 +173,22 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
  * Who needs it: code that must not call cudaMalloc — a serving process that has handed all device memory
  * to its framework's pool, a plug-in that only ever receives input and output pointers, anything that runs
  * where an allocation would synchronise the device or is forbidden.  kvq_attn_corrected needs a caller
- * workspace when it splits the key tiles of a unit over several CTAs (few query rows, long cache); this
- * entry point keeps those partial results in a scratch buffer that is part of the library image instead:
- * 64 slots of 134 144 bytes = 8 585 216 bytes of device memory on every GPU that loads libkvq.so, held
- * until the process exits.  It calls no allocating routine of CUDA or of any other library.
+ * workspace for the rotated query chunk and, when it splits the key tiles of a unit over several CTAs (few
+ * query rows, long cache), for their partial results; this entry point keeps both in a scratch buffer that
+ * is part of the library image instead: 8192 query rows of 272 bytes plus 64 slots of 134 144 bytes =
+ * 10 813 440 bytes of device memory on every GPU that loads libkvq.so, held until the process exits.  It
+ * calls no allocating routine of CUDA or of any other library.
  *
- * Limits: head_dim 128 only (the tcgen05 kernel; no kernel-selection flags).  A problem whose units
- * (batch * heads * ceil(m_tokens / 256)) are fewer than half the SMs is split, on at most 32 CTAs, and may
- * then have at most 32 units: more returns KVQ_ERR_WORKSPACE.  Larger problems are not split, use no
- * scratch and are accepted at any size.
+ * Limits: head_dim 128 only (the tcgen05 kernel; no kernel-selection flags).  Over a non-empty cache window
+ * batch * heads * m_tokens may be at most 8192 query rows.  A problem with fewer units (batch * heads *
+ * ceil(m_tokens / 256)) than SMs whose idle SMs are worth splitting for is split, on at most 32 CTAs, and
+ * may then have at most 32 units.  Beyond either limit the call returns KVQ_ERR_WORKSPACE and launches
+ * nothing.
  *
  * The first call on a device looks up the buffer's device address (cudaGetSymbolAddress, with that device
  * current) and remembers it; make that first call outside any stream capture.
  * All calls on a device share the one buffer and it keeps the previous call's contents.  Nothing in it has
- * to start at zero (every slot is written in full before it is read), so no clearing is done; but two calls
+ * to start at zero (every row and slot is written in full before it is read), so no clearing is done; but two calls
  * whose kernels overlap on the GPU (different streams, no ordering between them) race on it: order them.
  *
  * Arguments, outputs and the other error codes are those of kvq_attn_corrected, without the workspace.

@@ -92,6 +92,7 @@ struct TParams {
   int q_blocks, n_units, tiles;
   int n_whole;             // units [0, n_whole) are computed whole; the rest are split over all CTAs
   float* partial;          // workspace: 2 slots per CTA, see kSlotFloats
+  const uint16_t* ax_rows; // workspace: bias operand rows written by rotate_query_kernel, [batch*heads][m_tokens][8]
 };
 
 // One partial result: unnormalised O [256][128] FP32, then m[256], l_cur[256], l_cached[256]
@@ -359,84 +360,109 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
   }
 }
 
-// Rotates the CTA's 256-row query tile in place (four warps; 16 lanes per row, 8 channels per lane):
-// q~ = (1/sqrt d) H (signs . q) in FP32, written back as FP16 with the contraction dimension permuted the
-// way the dequantized keys are laid out, and -(sigma/24) nu_{m,j} written to the bias operand tile.
+// Pre-pass over the query chunk (one launch before the attention kernel): q~ = (1/sqrt d) H (signs . q) in
+// FP32, stored as FP16 with the contraction dimension permuted the way the dequantized keys are laid out,
+// and -(sigma/24) nu_{m,j} (per-group squared norms of q~) as a BF16 high part plus a BF16 low part.  The
+// attention kernel swaps the rotated tile in by TMA once the current chunk's score MMAs are done, so units
+// split over several CTAs rotate their rows once instead of once per CTA.
+// 16 lanes per row, 8 channels per lane; a warp handles two rows at a time, a block of 4 warps 64 rows.
+struct RotParams {
+  const uint16_t* q; int64_t q_sb, q_sh, q_st;
+  uint16_t* qr;            // [batch * heads][m_tokens][128] FP16
+  uint16_t* ax;            // [batch * heads][m_tokens][8] BF16: high parts of groups 0..3, then low parts
+  const int8_t* signs;
+  int heads, m_tokens, rotate;
+  float ax_coef;           // -sigma / 24
+};
+
 template <int BITS, int GROUP>
-__device__ __forceinline__ void rotate_query(uint8_t* smem, const TParams& p, int warp, int lane) {
-    const int l16 = lane & 15, rsub = lane >> 4;
-    constexpr int lanes_per_group = GROUP / 8;
-    float sgn[8];
+__global__ void __launch_bounds__(128) rotate_query_kernel(const RotParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int l16 = lane & 15, rsub = lane >> 4;
+  constexpr int lanes_per_group = GROUP / 8;
+  const int bh = blockIdx.y, b = bh / p.heads, h = bh - b * p.heads;
+  float sgn[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) sgn[e] = (p.rotate && p.signs) ? (float)p.signs[l16 * 8 + e] : 1.0f;
-    for (int pass = 0; pass < 32; ++pass) {
-      const int qrow = pass * 8 + (warp - 12) * 2 + rsub;     // 0..255
-      const int qt = qrow >> 7, rr = qrow & 127;
-      uint8_t* qtile = smem + kOffQ + qt * kTileBytes;
-      const uint4 raw = *reinterpret_cast<const uint4*>(qtile + sw128_offset(rr, l16));
-      float x[8];
-      x[0] = bf16_bits_to_f32(raw.x & 0xFFFFu); x[1] = bf16_bits_to_f32(raw.x >> 16);
-      x[2] = bf16_bits_to_f32(raw.y & 0xFFFFu); x[3] = bf16_bits_to_f32(raw.y >> 16);
-      x[4] = bf16_bits_to_f32(raw.z & 0xFFFFu); x[5] = bf16_bits_to_f32(raw.z >> 16);
-      x[6] = bf16_bits_to_f32(raw.w & 0xFFFFu); x[7] = bf16_bits_to_f32(raw.w >> 16);
-      if (p.rotate) {
+  for (int e = 0; e < 8; ++e) sgn[e] = (p.rotate && p.signs) ? (float)p.signs[l16 * 8 + e] : 1.0f;
+  for (int pass = 0; pass < 8; ++pass) {
+    const int row = blockIdx.x * 64 + pass * 8 + warp * 2 + rsub;
+    const bool valid = row < p.m_tokens;             // no early exit: the shuffles below need every lane
+    uint4 raw = make_uint4(0, 0, 0, 0);
+    if (valid) raw = __ldg(reinterpret_cast<const uint4*>(p.q + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + (int64_t)row * p.q_st) + l16);
+    float x[8];
+    x[0] = bf16_bits_to_f32(raw.x & 0xFFFFu); x[1] = bf16_bits_to_f32(raw.x >> 16);
+    x[2] = bf16_bits_to_f32(raw.y & 0xFFFFu); x[3] = bf16_bits_to_f32(raw.y >> 16);
+    x[4] = bf16_bits_to_f32(raw.z & 0xFFFFu); x[5] = bf16_bits_to_f32(raw.z >> 16);
+    x[6] = bf16_bits_to_f32(raw.w & 0xFFFFu); x[7] = bf16_bits_to_f32(raw.w >> 16);
+    if (p.rotate) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] *= sgn[e];
+      for (int e = 0; e < 8; ++e) x[e] *= sgn[e];
 #pragma unroll
-        for (int hh = 1; hh < 8; hh *= 2)
+      for (int hh = 1; hh < 8; hh *= 2)
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            if ((i & hh) == 0) { const float a = x[i], c = x[i + hh]; x[i] = a + c; x[i + hh] = a - c; }
+        for (int i = 0; i < 8; ++i)
+          if ((i & hh) == 0) { const float a = x[i], c = x[i + hh]; x[i] = a + c; x[i + hh] = a - c; }
 #pragma unroll
-        for (int lm = 1; lm < 16; lm *= 2)
+      for (int lm = 1; lm < 16; lm *= 2)
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
-            x[e] = (l16 & lm) ? (o - x[e]) : (x[e] + o);
-          }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] *= 0.08838834764831845f;
-      }
-      float nu = 0.f;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) nu += x[e] * x[e];
-      for (int off = 1; off < lanes_per_group; off *= 2) nu += __shfl_xor_sync(0xFFFFFFFFu, nu, off);
-      if ((l16 % lanes_per_group) == 0) {
-        const int j = l16 / lanes_per_group;
-        // -(sigma/24) nu as a BF16 high part plus a BF16 low part (columns j and 4 + j)
-        const float a = p.ax_coef * nu;
-        const uint32_t hi = f32_to_bf16_bits(a);
-        uint8_t* ax = smem + kOffAx + qt * kXBytes + xtile_offset(rr, 0);
-        *reinterpret_cast<uint16_t*>(ax + 2 * j) = (uint16_t)hi;
-        *reinterpret_cast<uint16_t*>(ax + 8 + 2 * j) = (uint16_t)f32_to_bf16_bits(a - bf16_bits_to_f32(hi));
-      }
-      float y[8];
-      if constexpr (BITS == 2) {
-        // physical column 16w + 2i + hsel <- channel 16w + i + 8*hsel: even lanes own the low half
-        // of a 16-channel word, odd lanes the high half; swap four values with the neighbour
-        const bool odd = l16 & 1;
-        float rcv[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) rcv[i] = __shfl_xor_sync(0xFFFFFFFFu, odd ? x[i] : x[4 + i], 1);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          y[2 * i] = odd ? rcv[i] : x[i];
-          y[2 * i + 1] = odd ? x[4 + i] : rcv[i];
+        for (int e = 0; e < 8; ++e) {
+          const float o = __shfl_xor_sync(0xFFFFFFFFu, x[e], lm);
+          x[e] = (l16 & lm) ? (o - x[e]) : (x[e] + o);
         }
-      } else {
-        // physical column 8w + 2i + hsel <- channel 8w + i + 4*hsel
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { y[2 * i] = x[i]; y[2 * i + 1] = x[4 + i]; }
-      }
-      *reinterpret_cast<uint4*>(qtile + sw128_offset(rr, l16)) =
-          make_uint4(pack_f16x2_sat(y[0], y[1]), pack_f16x2_sat(y[2], y[3]), pack_f16x2_sat(y[4], y[5]), pack_f16x2_sat(y[6], y[7]));
+      for (int e = 0; e < 8; ++e) x[e] *= 0.08838834764831845f;
     }
+    float nu = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) nu += x[e] * x[e];
+    for (int off = 1; off < lanes_per_group; off *= 2) nu += __shfl_xor_sync(0xFFFFFFFFu, nu, off);
+    {
+      // -(sigma/24) nu_j as a BF16 high part plus a BF16 low part: columns j and 4 + j of the row's 16 bytes,
+      // zeros for groups the format does not have; gathered from the group leaders and written by lane 0 of the row
+      const float a = p.ax_coef * nu;
+      const uint32_t hi = f32_to_bf16_bits(a);
+      const uint32_t lo = f32_to_bf16_bits(a - bf16_bits_to_f32(hi));
+      uint32_t h4[4], l4[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int src = (lane & 16) + ((j * lanes_per_group) & 15);
+        const uint32_t hj = __shfl_sync(0xFFFFFFFFu, hi, src), lj = __shfl_sync(0xFFFFFFFFu, lo, src);
+        const bool have = j * GROUP < kD;
+        h4[j] = have ? hj : 0u; l4[j] = have ? lj : 0u;
+      }
+      if (valid && l16 == 0)
+        *reinterpret_cast<uint4*>(p.ax + ((int64_t)bh * p.m_tokens + row) * 8) =
+            make_uint4(h4[0] | (h4[1] << 16), h4[2] | (h4[3] << 16), l4[0] | (l4[1] << 16), l4[2] | (l4[3] << 16));
+    }
+    float y[8];
+    if constexpr (BITS == 2) {
+      // physical column 16w + 2i + hsel <- channel 16w + i + 8*hsel: even lanes own the low half
+      // of a 16-channel word, odd lanes the high half; swap four values with the neighbour
+      const bool odd = l16 & 1;
+      float rcv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) rcv[i] = __shfl_xor_sync(0xFFFFFFFFu, odd ? x[i] : x[4 + i], 1);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        y[2 * i] = odd ? rcv[i] : x[i];
+        y[2 * i + 1] = odd ? x[4 + i] : rcv[i];
+      }
+    } else {
+      // physical column 8w + 2i + hsel <- channel 8w + i + 4*hsel
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { y[2 * i] = x[i]; y[2 * i + 1] = x[4 + i]; }
+    }
+    if (valid)
+      *(reinterpret_cast<uint4*>(p.qr + ((int64_t)bh * p.m_tokens + row) * kD) + l16) =
+        make_uint4(pack_f16x2_sat(y[0], y[1]), pack_f16x2_sat(y[2], y[3]), pack_f16x2_sat(y[4], y[5]), pack_f16x2_sat(y[6], y[7]));
+  }
 }
+
 
 template <int BITS, int GROUP>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, const TParams p) {
+attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qr,
+                    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -462,14 +488,14 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_init(cx.bar(kODone + s), 1);
     }
     mbar_init(cx.bar(kQCurDone), 1);
-    mbar_init(cx.bar(kQRotFull), 128);
+    mbar_init(cx.bar(kQRotFull), 129);   // 128 dequant threads (bias rows) + the TMA thread (rotated query tile)
     mbar_init(cx.bar(kDrain), 1);
     mbar_init(cx.bar(kQEmpty), 1);
     mbar_init(cx.bar(kOFree + 0), 256);
     mbar_init(cx.bar(kOFree + 1), 256);
     for (int i = 0; i < 8; ++i) mbar_init(cx.bar(kPair + i), 64);
     fence_barrier_init();
-    prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+    prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_qr); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
   }
   // bias operand tiles start as zeros (columns beyond the group count stay zero for good)
   for (int i = tid; i < 4 * kXBytes / 16; i += kThreads)
@@ -492,20 +518,32 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (lane == 0) {
       Schedule sch(blockIdx.x, gridDim.x, p);
       Segment sg;
-      int it = 0, nseg = 0, issued_it = -1;
+      int it = 0, nseg = 0, issued_it = -1, rot_seg = -1;
       bool ok = true;
       while (ok && sch.next(sg)) {
         const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
         const int row0 = (sg.unit - bh * p.q_blocks) * (2 * kBlockM);
         // the query buffer is free once every score MMA of the previous segment has retired
         if (!(ok = cx.wait(kQEmpty, (nseg & 1) ^ 1, 100))) break;
+        // a segment that starts in the cache never needs the unrotated query: load the rotated one right away
+        const bool cached0 = sg.tb >= n_rt;
         mbar_arrive_expect_tx(cx.bar(kQFull), 2 * kTileBytes);
         for (int qt = 0; qt < 2; ++qt)
           for (int kb = 0; kb < 2; ++kb)
-            tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, &tm_q, cx.bar(kQFull), kb * 64, row0 + qt * kBlockM, h, b);
+            tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, cached0 ? &tm_qr : &tm_q, cx.bar(kQFull), kb * 64, row0 + qt * kBlockM, h, b);
+        if (cached0 || sg.te <= n_rt) mbar_arrive(cx.bar(kQRotFull));   // this thread's share of the phase
         for (int t = sg.tb; t < sg.te; ++t, ++it) {
           const int s = it & 1;
           const uint32_t ph = (it >> 1) & 1;
+          if (t == n_rt && !cached0) {
+            // first cached tile: once no MMA reads the unrotated query any more, the rotated tile replaces it
+            if (!(ok = cx.wait(kQCurDone, nseg & 1, 103))) break;
+            mbar_arrive_expect_tx(cx.bar(kQRotFull), 2 * kTileBytes);
+            for (int qt = 0; qt < 2; ++qt)
+              for (int kb = 0; kb < 2; ++kb)
+                tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, &tm_qr, cx.bar(kQRotFull), kb * 64, row0 + qt * kBlockM, h, b);
+            rot_seg = nseg;
+          }
           if (!(ok = cx.wait(kKEmpty + s, ph ^ 1, 101))) break;
           if (t < n_rt) {
             mbar_arrive_expect_tx(cx.bar(kKFull + s), kTileBytes);
@@ -528,6 +566,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       if (*cx.abort) {   // drain: give loads already in flight a bounded time to land before the CTA exits
         if (nseg > 0) cx.drain(kQFull, (nseg - 1) & 1);
+        if (rot_seg >= 0) cx.drain(kQRotFull, rot_seg & 1);
         if (issued_it >= 0) {
           cx.drain(kKFull + (issued_it & 1), (issued_it >> 1) & 1);
           cx.drain(kVFull + (issued_it & 1), (issued_it >> 1) & 1);
@@ -844,10 +883,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         mbar_arrive(cx.bar(kKFull + s));
         if (t == t_rot) {
-          // ---- rotate the query tile in place; per-group squared norms -> A_extra ----
-          ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, nseg & 1, 402) && cx.wait(kQCurDone, nseg & 1, 403));
+          // ---- A_extra: -(sigma/24) nu rows of this unit's 256 queries, written by the pre-pass ----
+          // (the new query tile being in means every MMA of the previous segment, which read the old rows, retired)
+          ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, nseg & 1, 402));
           if (!ok) break;
-          rotate_query<BITS, GROUP>(smem, p, warp, lane);
+          const int row0 = (sg.unit - bh * p.q_blocks) * (2 * kBlockM);
+#pragma unroll
+          for (int qt = 0; qt < 2; ++qt) {
+            const int row = row0 + qt * kBlockM + dt;
+            uint4 a = make_uint4(0, 0, 0, 0);
+            if (row < p.m_tokens) a = __ldg(reinterpret_cast<const uint4*>(p.ax_rows + ((int64_t)bh * p.m_tokens + row) * 8));
+            *reinterpret_cast<uint4*>(smem + kOffAx + qt * kXBytes + xtile_offset(dt, 0)) = a;
+          }
           fence_proxy_async_smem();
           mbar_arrive(cx.bar(kQRotFull));
         }
@@ -979,10 +1026,10 @@ int num_sms() {
 //  * At least as many units as SMs: one persistent CTA per SM.  Whole units are dealt out in rounds of
 //    one per CTA; the last, incomplete round of R units would leave SMs idle for a whole unit's time, so
 //    when R is at most half the SMs its key-tile steps are split evenly over all CTAs instead.
-//  * Between half as many and as many units as SMs: one CTA per unit, nothing split (splitting measured
-//    slower than the idle SMs cost).
-//  * Fewer (short query chunk, long cache): all tile steps are cut into equal ranges, one per CTA, each at
-//    least ~4 tiles long.
+//  * Fewer units than SMs: one CTA per unit leaves sms - n_units SMs idle for `tiles` tile steps each.
+//    Cutting all tile steps into equal ranges, one per SM, uses them, at a measured cost of about ten
+//    tile steps per CTA (a second prologue and epilogue, FP32 partial results, the merge kernel): split
+//    when the idle time is worth more than that.
 struct Plan { int ctas; int n_whole; };
 Plan plan_grid(int64_t n_units, int64_t tiles) {
   const int sms = num_sms();
@@ -990,7 +1037,7 @@ Plan plan_grid(int64_t n_units, int64_t tiles) {
     const int64_t r = n_units % sms;
     return {sms, (int)((r == 0 || 2 * r > sms) ? n_units : n_units - r)};
   }
-  if (2 * n_units >= sms) return {(int)n_units, (int)n_units};
+  if (tiles * (sms - n_units) <= 10 * (int64_t)sms) return {(int)n_units, (int)n_units};
   const int64_t W = n_units * tiles;
   int64_t c = W / 4;
   if (c < n_units) c = n_units;
@@ -1000,13 +1047,18 @@ Plan plan_grid(int64_t n_units, int64_t tiles) {
 }
 
 template <int BITS, int GROUP>
-int launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TParams& p, dim3 grid, cudaStream_t st) {
+int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk, const CUtensorMap& mv, const TParams& p,
+           const RotParams& rp, dim3 grid, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_tcgen05_kernel<BITS, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured = true;
   }
-  attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
+  if (rp.qr) {                      // there are cached keys: rotate the query chunk first
+    rotate_query_kernel<BITS, GROUP><<<dim3((unsigned)((rp.m_tokens + 63) / 64), (unsigned)(p.n_units / p.q_blocks)), 128, 0, st>>>(rp);
+    KVQ_CUDA_TRY(cudaGetLastError());
+  }
+  attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mqr, mk, mv, p);
   KVQ_CUDA_TRY(cudaGetLastError());
   if (p.n_whole != p.n_units) {   // units were split over CTAs: combine their partial results
     attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 32), 128, 0, st>>>(p, (int)grid.x);
@@ -1028,23 +1080,47 @@ static void schedule_shape(const kvq_cache_desc* d, int64_t cache_len, int64_t m
   *tiles = (n_cur + kBlockN - 1) / kBlockN + (cache_len + kBlockN - 1) / kBlockN;
 }
 
+// Bytes of the rotated-query area of the workspace: q~ rows (256 bytes each), then bias rows (16 bytes each),
+// rounded up to a multiple of 256.  Nothing when there are no cached keys.
+static size_t rot_area_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens) {
+  if (cache_len <= 0) return 0;
+  const size_t rows = (size_t)d->batch * d->heads * (size_t)m_tokens;
+  return (rows * (2 * kD + 16) + 255) / 256 * 256;
+}
+
 size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur) {
   if (m_tokens <= 0) return 0;
   int64_t qb, nu, tiles;
   schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
   const Plan pl = plan_grid(nu, tiles);
-  return pl.n_whole != nu ? (size_t)pl.ctas * 2 * kSlotFloats * sizeof(float) : 0;
+  const size_t slots = pl.n_whole != nu ? (size_t)pl.ctas * 2 * kSlotFloats * sizeof(float) : 0;
+  return rot_area_bytes(d, cache_len, m_tokens) + slots;
 }
 
-int launch_attn_tcgen05(const AttnArgs& a) {
+// Common tail of both entry points.  `rot_area` (rot_area_bytes() bytes, 256-byte aligned; null only when
+// there are no cached keys) receives the rotated queries; `slots` holds the partial results of split units.
+static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, float* slots) {
   const kvq_cache_desc* d = a.desc;
   EncodeTiledFn enc;
   int r = get_encode_fn(&enc);
   if (r != KVQ_OK) return r;
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq, mqr, mk, mv;
   if ((r = make_map(enc, &mq, a.q, a.qs, a.m_tokens, d->heads, d->batch)) != KVQ_OK) return r;
   if ((r = make_map(enc, &mk, a.k_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
   if ((r = make_map(enc, &mv, a.v_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
+  RotParams rp{};
+  mqr = mq;                                                  // never read when there are no cached keys
+  if (rot_area) {
+    const int64_t rows = (int64_t)d->batch * d->heads * a.m_tokens;
+    rp.q = static_cast<const uint16_t*>(a.q); rp.q_sb = a.qs.b; rp.q_sh = a.qs.h; rp.q_st = a.qs.t;
+    rp.qr = reinterpret_cast<uint16_t*>(rot_area);
+    rp.ax = reinterpret_cast<uint16_t*>(rot_area + (size_t)rows * 2 * kD);
+    rp.signs = d->signs;
+    rp.heads = d->heads; rp.m_tokens = (int)a.m_tokens; rp.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
+    rp.ax_coef = -a.softmax_scale / 24.0f;
+    const kvq_strides dense{(int64_t)d->heads * a.m_tokens * kD, a.m_tokens * (int64_t)kD, (int64_t)kD};
+    if ((r = make_map(enc, &mqr, rp.qr, dense, a.m_tokens, d->heads, d->batch)) != KVQ_OK) return r;
+  }
   TParams p;
   p.out = static_cast<uint16_t*>(a.out); p.o_sb = a.os.b; p.o_sh = a.os.h; p.o_st = a.os.t;
   p.k_codes = static_cast<const uint8_t*>(d->k_codes); p.v_codes = static_cast<const uint8_t*>(d->v_codes);
@@ -1058,22 +1134,30 @@ int launch_attn_tcgen05(const AttnArgs& a) {
   p.scale_log2 = a.softmax_scale * kLog2e;
   p.ax_coef = -a.softmax_scale / 24.0f;
   p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
-  int64_t qb, nu, tiles;
-  schedule_shape(d, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
-  if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
   p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
-  p.partial = static_cast<float*>(a.workspace);
-  const Plan pl = plan_grid(nu, tiles);
+  p.partial = slots;
+  p.ax_rows = rp.ax;
   p.n_whole = pl.n_whole;
   dim3 grid((unsigned)pl.ctas);
   if (d->bits == 2) {
-    if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
-    if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);
-    return launch<2, 128>(mq, mk, mv, p, grid, a.stream);
+    if (d->group == 32) return launch<2, 32>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+    if (d->group == 64) return launch<2, 64>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+    return launch<2, 128>(mq, mqr, mk, mv, p, rp, grid, a.stream);
   }
-  if (d->group == 32) return launch<4, 32>(mq, mk, mv, p, grid, a.stream);
-  if (d->group == 64) return launch<4, 64>(mq, mk, mv, p, grid, a.stream);
-  return launch<4, 128>(mq, mk, mv, p, grid, a.stream);
+  if (d->group == 32) return launch<4, 32>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+  if (d->group == 64) return launch<4, 64>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+  return launch<4, 128>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+}
+
+int launch_attn_tcgen05(const AttnArgs& a) {
+  int64_t qb, nu, tiles;
+  schedule_shape(a.desc, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
+  if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
+  const Plan pl = plan_grid(nu, tiles);
+  // workspace: [rotated-query area][partial-result slots]; its size was checked by the caller
+  const size_t rot = rot_area_bytes(a.desc, a.cache_len, a.m_tokens);
+  uint8_t* ws = static_cast<uint8_t*>(a.workspace);
+  return launch_planned(a, pl, qb, nu, tiles, rot ? ws : nullptr, reinterpret_cast<float*>(ws + rot));
 }
 
 
@@ -1082,10 +1166,15 @@ int launch_attn_tcgen05(const AttnArgs& a) {
 // Some callers may not allocate device memory at all (an inference server that hands its whole memory pool
 // to a framework allocator up front, code running while a CUDA graph is being captured, a plug-in that is
 // only given input and output pointers).  For them the split-unit path can run on a scratch buffer that is
-// part of the library image: every GPU that loads libkvq.so carries these 8.2 MiB until the process exits.
+// part of the library image: every GPU that loads libkvq.so carries these 10.3 MiB until the process exits.
+// Layout: the rotated-query area for up to kStaticMaxRows query rows (batch * heads * m_tokens), then two
+// partial results for each of up to kStaticMaxCtas CTAs.
+constexpr int kStaticMaxRows = 8192;
 constexpr int kStaticMaxCtas = 32;                         // split problems run on at most this many CTAs
 constexpr int kStaticSlots = 2 * kStaticMaxCtas;           // two partial results per CTA
-static __device__ __align__(256) float g_static_scratch[(size_t)kStaticSlots * kSlotFloats];
+constexpr size_t kStaticRotFloats = (size_t)kStaticMaxRows * (2 * kD + 16) / 4;
+static_assert(kStaticRotFloats * 4 % 256 == 0, "slots must start 256-byte aligned");
+static __device__ __align__(256) float g_static_scratch[kStaticRotFloats + (size_t)kStaticSlots * kSlotFloats];
 
 // The array's name is only a host-side handle; the device address has to be asked for, once per device,
 // with that device current.
@@ -1111,50 +1200,26 @@ int launch_attn_tcgen05_static(const AttnArgs& a) {
   schedule_shape(d, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
   if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
   Plan pl = plan_grid(nu, tiles);
-  float* scratch = nullptr;
+  bool need_slots = false;
   if (pl.n_whole != nu) {
     if (pl.n_whole > 0) {
-      pl.n_whole = (int)nu;                                // many units: deal all of them out whole, no scratch
-    } else {                                               // few units, all split: partial results need the scratch
+      pl.n_whole = (int)nu;                                // many units: deal all of them out whole, no slots
+    } else {                                               // few units, all split: partial results need the slots
       if (nu > kStaticMaxCtas) return KVQ_ERR_WORKSPACE;   // stated maximum: 32 units when splitting
       if (pl.ctas > kStaticMaxCtas) pl.ctas = kStaticMaxCtas;
       if (pl.ctas < nu) pl.ctas = (int)nu;
-      const int r = static_scratch_ptr(&scratch);
-      if (r != KVQ_OK) return r;
+      need_slots = true;
     }
   }
-  EncodeTiledFn enc;
-  int r = get_encode_fn(&enc);
-  if (r != KVQ_OK) return r;
-  CUtensorMap mq, mk, mv;
-  if ((r = make_map(enc, &mq, a.q, a.qs, a.m_tokens, d->heads, d->batch)) != KVQ_OK) return r;
-  if ((r = make_map(enc, &mk, a.k_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
-  if ((r = make_map(enc, &mv, a.v_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
-  TParams p;
-  p.out = static_cast<uint16_t*>(a.out); p.o_sb = a.os.b; p.o_sh = a.os.h; p.o_st = a.os.t;
-  p.k_codes = static_cast<const uint8_t*>(d->k_codes); p.v_codes = static_cast<const uint8_t*>(d->v_codes);
-  p.k_scale = static_cast<const uint8_t*>(d->k_scale); p.v_scale = static_cast<const uint8_t*>(d->v_scale);
-  p.k_zero = static_cast<const uint16_t*>(d->k_zero); p.v_zero = static_cast<const uint16_t*>(d->v_zero);
-  p.signs = d->signs;
-  p.capacity = d->capacity; p.cache_begin = a.cache_begin;
-  p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
-  p.correction = (a.flags & KVQ_CORRECTION_ON) ? 1 : 0;
-  p.m_tokens = (int)a.m_tokens; p.n_cached = (int)a.cache_len; p.n_cur = (int)a.n_cur;
-  p.scale_log2 = a.softmax_scale * kLog2e;
-  p.ax_coef = -a.softmax_scale / 24.0f;
-  p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
-  p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
-  p.partial = scratch;
-  p.n_whole = pl.n_whole;
-  dim3 grid((unsigned)pl.ctas);
-  if (d->bits == 2) {
-    if (d->group == 32) return launch<2, 32>(mq, mk, mv, p, grid, a.stream);
-    if (d->group == 64) return launch<2, 64>(mq, mk, mv, p, grid, a.stream);
-    return launch<2, 128>(mq, mk, mv, p, grid, a.stream);
+  const size_t rot = rot_area_bytes(d, a.cache_len, a.m_tokens);
+  if (rot > kStaticRotFloats * 4) return KVQ_ERR_WORKSPACE;  // stated maximum: 8192 query rows over a non-empty cache
+  float* scratch = nullptr;
+  if (rot || need_slots) {
+    const int r = static_scratch_ptr(&scratch);
+    if (r != KVQ_OK) return r;
   }
-  if (d->group == 32) return launch<4, 32>(mq, mk, mv, p, grid, a.stream);
-  if (d->group == 64) return launch<4, 64>(mq, mk, mv, p, grid, a.stream);
-  return launch<4, 128>(mq, mk, mv, p, grid, a.stream);
+  return launch_planned(a, pl, qb, nu, tiles, rot ? reinterpret_cast<uint8_t*>(scratch) : nullptr,
+                        need_slots ? scratch + kStaticRotFloats : nullptr);
 }
 
 }  // namespace kvq

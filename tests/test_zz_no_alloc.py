@@ -61,18 +61,24 @@ def test_matches_workspace_entry_point_on_two_calls_in_a_row(B):
             assert np.abs(mass_st - mass_ws).max() < 1e-2
 
 
-def test_unsplit_problem_needs_no_scratch_and_is_identical(B):
-    g, q, kc, vc = _problem(B, heads=40, m=512, chunks=2, chunk_tokens=300, n_cur=256, seed=3)   # 80 units: one CTA each
-    assert B.kvq_attn_workspace_bytes(g, g.length, 512, 256, B.KVQ_CORRECTION_ON) == 0
+def test_unsplit_problem_uses_only_the_query_area_and_is_identical(B):
+    g, q, kc, vc = _problem(B, heads=80, m=100, chunks=2, chunk_tokens=300, n_cur=256, seed=3)   # 80 units: one CTA each
+    # no partial-result slots: the workspace is just the rotated queries (256 + 16 bytes per query row)
+    assert B.kvq_attn_workspace_bytes(g, g.length, 100, 256, B.KVQ_CORRECTION_ON) == 80 * 100 * 272
     (o_ws, _, _), (o_st, _, _) = _both(B, g, q, kc, vc, B.KVQ_CORRECTION_ON)
     assert np.array_equal(o_ws, o_st)
 
 
 def test_sizes_beyond_the_buffer_are_refused(B):
-    g, q, kc, vc = _problem(B, heads=40, m=100, chunks=2, chunk_tokens=300, n_cur=100, seed=4)   # 40 units, split
+    g, q, kc, vc = _problem(B, heads=40, m=100, chunks=2, chunk_tokens=2000, n_cur=100, seed=4)   # 40 units of 33 tiles: split
     out = torch.empty_like(q)
     with pytest.raises(B.KvqError) as e:
         B.kvq_attn_corrected_static_scratch(g, q, kc, vc, T.sigma_of(128), B.KVQ_CORRECTION_ON, out=out)
+    assert e.value.status == B.KVQ_ERR_WORKSPACE
+    # more than 8192 query rows over a non-empty cache: the rotated queries do not fit
+    g2, q2, k2, v2 = _problem(B, heads=40, m=512, chunks=2, chunk_tokens=300, n_cur=256, seed=5)
+    with pytest.raises(B.KvqError) as e:
+        B.kvq_attn_corrected_static_scratch(g2, q2, k2, v2, T.sigma_of(128), B.KVQ_CORRECTION_ON, out=torch.empty_like(q2))
     assert e.value.status == B.KVQ_ERR_WORKSPACE
     # head_dim 64 has no tcgen05 kernel, kernel-selection flags are not accepted
     w = inputs.Workload("noalloc64", 499, 1, 2, 64, 100, 0, 2, 64, 0)
