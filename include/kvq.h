@@ -175,8 +175,8 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
  * where an allocation would synchronise the device or is forbidden.  kvq_attn_corrected needs a caller
  * workspace for the rotated query chunk and, when it splits the key tiles of a unit over several CTAs (few
  * query rows, long cache), for their partial results; this entry point keeps both in a scratch buffer that
- * is part of the library image instead: 8192 query rows of 272 bytes plus 64 slots of 134 144 bytes =
- * 10 813 440 bytes of device memory on every GPU that loads libkvq.so, held until the process exits.  It
+ * is part of the library image instead: 8192 query rows of 272 bytes plus 64 slots of 68 608 bytes =
+ * 6 619 136 bytes of device memory on every GPU that loads libkvq.so, held until the process exits.  It
  * calls no allocating routine of CUDA or of any other library.
  *
  * Limits: head_dim 128 only (the tcgen05 kernel; no kernel-selection flags).  Over a non-empty cache window

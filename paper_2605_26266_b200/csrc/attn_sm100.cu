@@ -91,12 +91,15 @@ struct TParams {
   // schedule: units = (batch*head, 256-row query block); every unit has `tiles` key tiles (see Schedule)
   int q_blocks, n_units, tiles;
   int n_whole;             // units [0, n_whole) are computed whole; the rest are split over all CTAs
-  float* partial;          // workspace: 2 slots per CTA, see kSlotFloats
+  uint8_t* partial;        // workspace: 2 slots per CTA, see kSlotBytes
   const uint16_t* ax_rows; // workspace: bias operand rows written by rotate_query_kernel, [batch*heads][m_tokens][8]
 };
 
-// One partial result: unnormalised O [256][128] FP32, then m[256], l_cur[256], l_cached[256]
-constexpr int kSlotFloats = 256 * kD + 3 * 256;
+// One partial result: the segment's own normalised output O / l as BF16 [256][128], then FP32 m[256],
+// l_cur[256], l_cached[256] (running maximum in log2 units and the row sums over current and cached keys).
+constexpr int kSlotStats = 256 * kD * 2;
+constexpr int kSlotBytes = kSlotStats + 3 * 256 * 4;
+static_assert(kSlotBytes % 256 == 0, "slots stay 256-byte aligned");
 
 // A contiguous run of key tiles [tb, te) of one unit; `slot` is the CTA's partial-result slot if the run is
 // not the whole unit.
@@ -365,7 +368,8 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
 // and -(sigma/24) nu_{m,j} (per-group squared norms of q~) as a BF16 high part plus a BF16 low part.  The
 // attention kernel swaps the rotated tile in by TMA once the current chunk's score MMAs are done, so units
 // split over several CTAs rotate their rows once instead of once per CTA.
-// 16 lanes per row, 8 channels per lane; a warp handles two rows at a time, a block of 4 warps 64 rows.
+// 16 lanes per row, 8 channels per lane; a warp handles two rows, a block of 8 warps 16 rows (many small
+// blocks: the kernel is a chain of dependent shuffles per row, so it wants every row in flight at once).
 struct RotParams {
   const uint16_t* q; int64_t q_sb, q_sh, q_st;
   uint16_t* qr;            // [batch * heads][m_tokens][128] FP16
@@ -376,7 +380,7 @@ struct RotParams {
 };
 
 template <int BITS, int GROUP>
-__global__ void __launch_bounds__(128) rotate_query_kernel(const RotParams p) {
+__global__ void __launch_bounds__(256) rotate_query_kernel(const RotParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int l16 = lane & 15, rsub = lane >> 4;
   constexpr int lanes_per_group = GROUP / 8;
@@ -384,8 +388,8 @@ __global__ void __launch_bounds__(128) rotate_query_kernel(const RotParams p) {
   float sgn[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) sgn[e] = (p.rotate && p.signs) ? (float)p.signs[l16 * 8 + e] : 1.0f;
-  for (int pass = 0; pass < 8; ++pass) {
-    const int row = blockIdx.x * 64 + pass * 8 + warp * 2 + rsub;
+  {
+    const int row = blockIdx.x * 16 + warp * 2 + rsub;
     const bool valid = row < p.m_tokens;             // no early exit: the shuffles below need every lane
     uint4 raw = make_uint4(0, 0, 0, 0);
     if (valid) raw = __ldg(reinterpret_cast<const uint4*>(p.q + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + (int64_t)row * p.q_st) + l16);
@@ -787,7 +791,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // ---- segment epilogue: read O out of TMEM, release it, combine the two column halves' row sums ----
       const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
       const bool whole = sg.tb == 0 && sg.te == T;
-      float* slot = p.partial + (size_t)(2 * blockIdx.x + sg.slot) * kSlotFloats;   // partial segments only
+      uint8_t* slot = p.partial + (size_t)(2 * blockIdx.x + sg.slot) * kSlotBytes;   // partial segments only
 #pragma unroll 1
       for (int qt = 0; qt < 2; ++qt) {
         const int r256 = qt * kBlockM + r128;
@@ -808,35 +812,31 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const float lc = lcur_a + xl[((half ^ 1) * 256 + r256) * 2];
         const float la = lcac_a + xl[((half ^ 1) * 256 + r256) * 2 + 1];
         const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
-        if (whole) {
-          if (row < p.m_tokens) {
-            const float l = lc + la;
-            const float inv = 1.0f / l;
-            uint16_t* dst = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + half * 64;
+        // a whole unit writes its rows of the output; a partial segment writes the same normalised rows into its
+        // slot, with the statistics the merge kernel weighs them by
+        const float l = lc + la;
+        const float inv = 1.0f / l;
+        if (!whole || row < p.m_tokens) {
+          uint16_t* dst = whole ? p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + half * 64
+                                : reinterpret_cast<uint16_t*>(slot) + r256 * kD + half * 64;
 #pragma unroll
-            for (int i = 0; i < 64; i += 8) {
-              uint4 v;
-              v.x = cvt_bf16x2(__uint_as_float(sr[i]) * inv, __uint_as_float(sr[i + 1]) * inv);
-              v.y = cvt_bf16x2(__uint_as_float(sr[i + 2]) * inv, __uint_as_float(sr[i + 3]) * inv);
-              v.z = cvt_bf16x2(__uint_as_float(sr[i + 4]) * inv, __uint_as_float(sr[i + 5]) * inv);
-              v.w = cvt_bf16x2(__uint_as_float(sr[i + 6]) * inv, __uint_as_float(sr[i + 7]) * inv);
-              *reinterpret_cast<uint4*>(dst + i) = v;
-            }
-            if (half == 0) {
+          for (int i = 0; i < 64; i += 8) {
+            uint4 v;
+            v.x = cvt_bf16x2(__uint_as_float(sr[i]) * inv, __uint_as_float(sr[i + 1]) * inv);
+            v.y = cvt_bf16x2(__uint_as_float(sr[i + 2]) * inv, __uint_as_float(sr[i + 3]) * inv);
+            v.z = cvt_bf16x2(__uint_as_float(sr[i + 4]) * inv, __uint_as_float(sr[i + 5]) * inv);
+            v.w = cvt_bf16x2(__uint_as_float(sr[i + 6]) * inv, __uint_as_float(sr[i + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + i) = v;
+          }
+          if (half == 0) {
+            if (whole) {
               const int64_t idx = (int64_t)bh * p.m_tokens + row;
               if (p.lse) p.lse[idx] = (m_a + log2f(l)) * 0.6931471805599453f;
               if (p.cached_mass) p.cached_mass[idx] = la * inv;
+            } else {
+              float* st = reinterpret_cast<float*>(slot + kSlotStats);
+              st[r256] = m_a; st[256 + r256] = lc; st[512 + r256] = la;
             }
-          }
-        } else {
-          float4* orow = reinterpret_cast<float4*>(slot + (size_t)r256 * kD + half * 64);
-#pragma unroll
-          for (int i = 0; i < 64; i += 4)
-            orow[i >> 2] = make_float4(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1]), __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
-          if (half == 0) {
-            slot[256 * kD + r256] = m_a;
-            slot[256 * kD + 256 + r256] = lc;
-            slot[256 * kD + 512 + r256] = la;
           }
         }
         { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
@@ -927,16 +927,26 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_ctas) {
   const int unit = p.n_whole + blockIdx.x;
   const int T = p.tiles;
-  const long long W = (long long)(p.n_units - p.n_whole) * T;     // tile steps of the split part
-  const long long g_lo = (long long)blockIdx.x * T, g_hi = g_lo + T;
-  auto start = [&](long long c) { return W * c / n_ctas; };
-  auto owner = [&](long long g) {
-    long long c = g * n_ctas / W;
-    while (c + 1 < n_ctas && start(c + 1) <= g) ++c;
-    while (c > 0 && start(c) > g) --c;
-    return (int)c;
-  };
-  const int c_first = owner(g_lo), c_last = owner(g_hi - 1);
+  // Which CTAs worked on this unit, found once per block (64-bit divisions): CTA c owns the tile steps
+  // [W c / n_ctas, W (c + 1) / n_ctas) of the split part.  A CTA's slot 0 belongs to the unit its range starts
+  // in, slot 1 to the next one, so only the first CTA of a unit can have used slot 1 for it.
+  __shared__ int s_first, s_last, s_first_slot;
+  if (threadIdx.x == 0) {
+    const long long W = (long long)(p.n_units - p.n_whole) * T;     // tile steps of the split part
+    const long long g_lo = (long long)blockIdx.x * T, g_hi = g_lo + T;
+    auto start = [&](long long c) { return W * c / n_ctas; };
+    auto owner = [&](long long g) {
+      long long c = g * n_ctas / W;
+      while (c + 1 < n_ctas && start(c + 1) <= g) ++c;
+      while (c > 0 && start(c) > g) --c;
+      return (int)c;
+    };
+    s_first = owner(g_lo);
+    s_last = owner(g_hi - 1);
+    s_first_slot = start(s_first) >= g_lo ? 0 : 1;
+  }
+  __syncthreads();
+  const int c_first = s_first, c_last = s_last, first_slot = s_first_slot;
   if (c_first == c_last) return;                       // the unit was computed whole by one CTA
   const int r256 = blockIdx.y * 8 + (threadIdx.x >> 4);
   const int cg = threadIdx.x & 15;
@@ -945,21 +955,25 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_
   if (row >= p.m_tokens) return;
   float m = -INFINITY;
   for (int c = c_first; c <= c_last; ++c) {
-    const int slot = 2 * c + (p.n_whole + (int)(start(c) / T) == unit ? 0 : 1);
-    m = fmaxf(m, p.partial[(size_t)slot * kSlotFloats + 256 * kD + r256]);
+    const int slot = 2 * c + (c == c_first ? first_slot : 0);
+    m = fmaxf(m, reinterpret_cast<const float*>(p.partial + (size_t)slot * kSlotBytes + kSlotStats)[r256]);
   }
+  // out = sum_i w_i O_i / sum_i w_i with w_i = l_i 2^(m_i - m): every partial row is already normalised by its l_i
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   float l_cur = 0.f, l_cac = 0.f;
   for (int c = c_first; c <= c_last; ++c) {
-    const int slot = 2 * c + (p.n_whole + (int)(start(c) / T) == unit ? 0 : 1);
-    const float* sl = p.partial + (size_t)slot * kSlotFloats;
-    const float f = exp2f(sl[256 * kD + r256] - m);
-    l_cur += f * sl[256 * kD + 256 + r256];
-    l_cac += f * sl[256 * kD + 512 + r256];
-    const float4 a0 = *reinterpret_cast<const float4*>(sl + (size_t)r256 * kD + cg * 8);
-    const float4 a1 = *reinterpret_cast<const float4*>(sl + (size_t)r256 * kD + cg * 8 + 4);
-    acc[0] += f * a0.x; acc[1] += f * a0.y; acc[2] += f * a0.z; acc[3] += f * a0.w;
-    acc[4] += f * a1.x; acc[5] += f * a1.y; acc[6] += f * a1.z; acc[7] += f * a1.w;
+    const int slot = 2 * c + (c == c_first ? first_slot : 0);
+    const uint8_t* sl = p.partial + (size_t)slot * kSlotBytes;
+    const float* st = reinterpret_cast<const float*>(sl + kSlotStats);
+    const float f = exp2f(st[r256] - m);
+    const float lc = f * st[256 + r256], la = f * st[512 + r256];
+    l_cur += lc; l_cac += la;
+    const float w = lc + la;
+    const uint4 a = *reinterpret_cast<const uint4*>(sl + ((size_t)r256 * kD + cg * 8) * 2);
+    acc[0] += w * bf16_bits_to_f32(a.x & 0xFFFFu); acc[1] += w * bf16_bits_to_f32(a.x >> 16);
+    acc[2] += w * bf16_bits_to_f32(a.y & 0xFFFFu); acc[3] += w * bf16_bits_to_f32(a.y >> 16);
+    acc[4] += w * bf16_bits_to_f32(a.z & 0xFFFFu); acc[5] += w * bf16_bits_to_f32(a.z >> 16);
+    acc[6] += w * bf16_bits_to_f32(a.w & 0xFFFFu); acc[7] += w * bf16_bits_to_f32(a.w >> 16);
   }
   const float l = l_cur + l_cac, inv = 1.0f / l;
   uint4 v;
@@ -1055,7 +1069,7 @@ int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk,
     configured = true;
   }
   if (rp.qr) {                      // there are cached keys: rotate the query chunk first
-    rotate_query_kernel<BITS, GROUP><<<dim3((unsigned)((rp.m_tokens + 63) / 64), (unsigned)(p.n_units / p.q_blocks)), 128, 0, st>>>(rp);
+    rotate_query_kernel<BITS, GROUP><<<dim3((unsigned)((rp.m_tokens + 15) / 16), (unsigned)(p.n_units / p.q_blocks)), 256, 0, st>>>(rp);
     KVQ_CUDA_TRY(cudaGetLastError());
   }
   attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mqr, mk, mv, p);
@@ -1093,13 +1107,13 @@ size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, 
   int64_t qb, nu, tiles;
   schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
   const Plan pl = plan_grid(nu, tiles);
-  const size_t slots = pl.n_whole != nu ? (size_t)pl.ctas * 2 * kSlotFloats * sizeof(float) : 0;
+  const size_t slots = pl.n_whole != nu ? (size_t)pl.ctas * 2 * kSlotBytes : 0;
   return rot_area_bytes(d, cache_len, m_tokens) + slots;
 }
 
 // Common tail of both entry points.  `rot_area` (rot_area_bytes() bytes, 256-byte aligned; null only when
 // there are no cached keys) receives the rotated queries; `slots` holds the partial results of split units.
-static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, float* slots) {
+static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, uint8_t* slots) {
   const kvq_cache_desc* d = a.desc;
   EncodeTiledFn enc;
   int r = get_encode_fn(&enc);
@@ -1157,7 +1171,7 @@ int launch_attn_tcgen05(const AttnArgs& a) {
   // workspace: [rotated-query area][partial-result slots]; its size was checked by the caller
   const size_t rot = rot_area_bytes(a.desc, a.cache_len, a.m_tokens);
   uint8_t* ws = static_cast<uint8_t*>(a.workspace);
-  return launch_planned(a, pl, qb, nu, tiles, rot ? ws : nullptr, reinterpret_cast<float*>(ws + rot));
+  return launch_planned(a, pl, qb, nu, tiles, rot ? ws : nullptr, ws + rot);
 }
 
 
@@ -1166,21 +1180,21 @@ int launch_attn_tcgen05(const AttnArgs& a) {
 // Some callers may not allocate device memory at all (an inference server that hands its whole memory pool
 // to a framework allocator up front, code running while a CUDA graph is being captured, a plug-in that is
 // only given input and output pointers).  For them the split-unit path can run on a scratch buffer that is
-// part of the library image: every GPU that loads libkvq.so carries these 10.3 MiB until the process exits.
+// part of the library image: every GPU that loads libkvq.so carries these 6.3 MiB until the process exits.
 // Layout: the rotated-query area for up to kStaticMaxRows query rows (batch * heads * m_tokens), then two
 // partial results for each of up to kStaticMaxCtas CTAs.
 constexpr int kStaticMaxRows = 8192;
 constexpr int kStaticMaxCtas = 32;                         // split problems run on at most this many CTAs
 constexpr int kStaticSlots = 2 * kStaticMaxCtas;           // two partial results per CTA
-constexpr size_t kStaticRotFloats = (size_t)kStaticMaxRows * (2 * kD + 16) / 4;
-static_assert(kStaticRotFloats * 4 % 256 == 0, "slots must start 256-byte aligned");
-static __device__ __align__(256) float g_static_scratch[kStaticRotFloats + (size_t)kStaticSlots * kSlotFloats];
+constexpr size_t kStaticRotBytes = (size_t)kStaticMaxRows * (2 * kD + 16);
+static_assert(kStaticRotBytes % 256 == 0, "slots must start 256-byte aligned");
+static __device__ __align__(256) uint8_t g_static_scratch[kStaticRotBytes + (size_t)kStaticSlots * kSlotBytes];
 
 // The array's name is only a host-side handle; the device address has to be asked for, once per device,
 // with that device current.
-static int static_scratch_ptr(float** out) {
+static int static_scratch_ptr(uint8_t** out) {
   constexpr int kMaxDevices = 64;
-  static float* ptrs[kMaxDevices] = {};
+  static uint8_t* ptrs[kMaxDevices] = {};
   int dev = 0;
   KVQ_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return KVQ_ERR_UNSUPPORTED;
@@ -1188,7 +1202,7 @@ static int static_scratch_ptr(float** out) {
     void* p = nullptr;
     KVQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
     if (!p) return record_cuda_error(cudaErrorInvalidSymbol);
-    ptrs[dev] = static_cast<float*>(p);
+    ptrs[dev] = static_cast<uint8_t*>(p);
   }
   *out = ptrs[dev];
   return KVQ_OK;
@@ -1212,14 +1226,13 @@ int launch_attn_tcgen05_static(const AttnArgs& a) {
     }
   }
   const size_t rot = rot_area_bytes(d, a.cache_len, a.m_tokens);
-  if (rot > kStaticRotFloats * 4) return KVQ_ERR_WORKSPACE;  // stated maximum: 8192 query rows over a non-empty cache
-  float* scratch = nullptr;
+  if (rot > kStaticRotBytes) return KVQ_ERR_WORKSPACE;  // stated maximum: 8192 query rows over a non-empty cache
+  uint8_t* scratch = nullptr;
   if (rot || need_slots) {
     const int r = static_scratch_ptr(&scratch);
     if (r != KVQ_OK) return r;
   }
-  return launch_planned(a, pl, qb, nu, tiles, rot ? reinterpret_cast<uint8_t*>(scratch) : nullptr,
-                        need_slots ? scratch + kStaticRotFloats : nullptr);
+  return launch_planned(a, pl, qb, nu, tiles, rot ? scratch : nullptr, need_slots ? scratch + kStaticRotBytes : nullptr);
 }
 
 }  // namespace kvq
