@@ -934,16 +934,18 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_
   if (threadIdx.x == 0) {
     const long long W = (long long)(p.n_units - p.n_whole) * T;     // tile steps of the split part
     const long long g_lo = (long long)blockIdx.x * T, g_hi = g_lo + T;
-    auto start = [&](long long c) { return W * c / n_ctas; };
+    // floor(W c / n) <= g  <=>  W c < (g + 1) n: the exact tests need no division, a double gives the first guess
+    auto starts_by = [&](long long c, long long g) { return W * c < (g + 1) * n_ctas; };
     auto owner = [&](long long g) {
-      long long c = g * n_ctas / W;
-      while (c + 1 < n_ctas && start(c + 1) <= g) ++c;
-      while (c > 0 && start(c) > g) --c;
+      long long c = (long long)((double)g * n_ctas / (double)W);
+      c = c < 0 ? 0 : (c > n_ctas - 1 ? n_ctas - 1 : c);
+      while (c + 1 < n_ctas && starts_by(c + 1, g)) ++c;
+      while (c > 0 && !starts_by(c, g)) --c;
       return (int)c;
     };
     s_first = owner(g_lo);
     s_last = owner(g_hi - 1);
-    s_first_slot = start(s_first) >= g_lo ? 0 : 1;
+    s_first_slot = W * s_first >= g_lo * n_ctas ? 0 : 1;       // its range starts in this unit
   }
   __syncthreads();
   const int c_first = s_first, c_last = s_last, first_slot = s_first_slot;
