@@ -302,7 +302,9 @@ def main():
                          "peak_kind": ("burst" if bursty else "sustained") + " bf16, " + peaks["source"],
                          "frac_of_sustained": attn_tf / peaks["tf_sustained"],
                          "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
-            "gpu_launches": 2 * args.steps,
+            # kernels of this library launched inside the timed region: per step the attention call's
+            # (pre-pass, attention, merge as the problem needs them) plus one quantize-append
+            "gpu_launches": (B.kvq_attn_kernel_launches(cache, n_cached, q.shape[2], k.shape[2], flags) + 1) * args.steps,
             "clocks": clocks,
         }
         if not args.no_e2e:

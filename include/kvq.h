@@ -126,6 +126,15 @@ int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len,
                              int64_t m_tokens, int64_t n_cur, uint32_t flags, size_t* out_bytes);
 
 /*
+ * How many kernels one kvq_attn_corrected call launches for this problem (host-side bookkeeping for
+ * benchmarks and launch-bound callers): the attention kernel, the query pre-pass when the cache window
+ * is not empty, the merge kernel when units are split over CTAs.  out_count is host memory.  Same
+ * argument checks and errors as kvq_attn_workspace_bytes.
+ */
+int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len,
+                             int64_t m_tokens, int64_t n_cur, uint32_t flags, int* out_count);
+
+/*
  * Corrected chunk attention (paper Algorithm 1; Eqs. (2)-(4) for scores, partition sums and
  * cached mass; Eq. (15) and its rotated form Eq. (25) for the bias; Sec. 4.2: the bias is
  * subtracted from cached scores only).

@@ -58,6 +58,9 @@ def _load():
     lib.kvq_attn_workspace_bytes.restype = C.c_int
     lib.kvq_attn_workspace_bytes.argtypes = [C.POINTER(kvq_cache_desc), C.c_int64, C.c_int64, C.c_int64,
                                              C.c_uint32, C.POINTER(C.c_size_t)]
+    lib.kvq_attn_kernel_launches.restype = C.c_int
+    lib.kvq_attn_kernel_launches.argtypes = [C.POINTER(kvq_cache_desc), C.c_int64, C.c_int64, C.c_int64,
+                                             C.c_uint32, C.POINTER(C.c_int)]
     lib.kvq_attn_corrected.restype = C.c_int
     lib.kvq_attn_corrected.argtypes = [
         C.POINTER(kvq_cache_desc), C.c_int64, C.c_int64,
@@ -166,6 +169,13 @@ def kvq_attn_workspace_bytes(cache: Cache, cache_len: int, m_tokens: int, n_cur:
     out = C.c_size_t(0)
     _check(lib.kvq_attn_workspace_bytes(C.byref(cache.desc), cache_len, m_tokens, n_cur, flags, C.byref(out)),
            "kvq_attn_workspace_bytes")
+    return out.value
+
+
+def kvq_attn_kernel_launches(cache: Cache, cache_len: int, m_tokens: int, n_cur: int, flags: int) -> int:
+    out = C.c_int(0)
+    _check(lib.kvq_attn_kernel_launches(C.byref(cache.desc), cache_len, m_tokens, n_cur, flags, C.byref(out)),
+           "kvq_attn_kernel_launches")
     return out.value
 
 

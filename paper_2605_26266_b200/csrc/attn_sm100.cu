@@ -1113,6 +1113,14 @@ size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, 
   return rot_area_bytes(d, cache_len, m_tokens) + slots;
 }
 
+int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur) {
+  if (m_tokens <= 0) return 0;
+  int64_t qb, nu, tiles;
+  schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
+  const Plan pl = plan_grid(nu, tiles);
+  return 1 + (cache_len > 0 ? 1 : 0) + (pl.n_whole != nu ? 1 : 0);   // attention, query pre-pass, merge
+}
+
 // Common tail of both entry points.  `rot_area` (rot_area_bytes() bytes, 256-byte aligned; null only when
 // there are no cached keys) receives the rotated queries; `slots` holds the partial results of split units.
 static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, uint8_t* slots) {

@@ -125,6 +125,18 @@ int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len, int6
   return KVQ_OK;
 }
 
+int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len, int64_t m_tokens,
+                             int64_t n_cur, uint32_t flags, int* out_count) {
+  if (!out_count) return KVQ_ERR_INVALID_ARG;
+  int r = check_attn_args(desc, 0, cache_len, m_tokens, n_cur, flags);
+  if (r != KVQ_OK) return r;
+  int err;
+  const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
+  if (err != KVQ_OK) return err;
+  *out_count = tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur) : (m_tokens > 0 ? 1 : 0);
+  return KVQ_OK;
+}
+
 int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
                        const void* q, kvq_strides q_strides, const void* k_cur, const void* v_cur,
                        kvq_strides kv_strides, int64_t m_tokens, int64_t n_cur, void* out_bf16,

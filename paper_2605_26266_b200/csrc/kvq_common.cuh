@@ -50,6 +50,7 @@ int launch_attn_mma_sync(const AttnArgs& a);
 // tcgen05 kernel: returns KVQ_ERR_UNSUPPORTED for shapes it does not cover.
 bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur);
 size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
+int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
 int launch_attn_tcgen05(const AttnArgs& a);
 // Same kernel, partial results of split units in the library's built-in scratch buffer (no caller workspace).
 int launch_attn_tcgen05_static(const AttnArgs& a);

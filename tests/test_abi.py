@@ -26,7 +26,7 @@ def declared_symbols():
 def test_header_symbols_exported(binding):
     syms = declared_symbols()
     assert {"kvq_quantize_append", "kvq_attn_corrected", "kvq_cache_bytes", "kvq_unpack_codes",
-            "kvq_attn_workspace_bytes", "kvq_status_string", "kvq_last_cuda_error", "kvq_version"} <= set(syms)
+            "kvq_attn_workspace_bytes", "kvq_attn_kernel_launches", "kvq_status_string", "kvq_last_cuda_error", "kvq_version"} <= set(syms)
     for s in syms:
         assert hasattr(binding.lib, s), s
 
