@@ -81,44 +81,57 @@ __device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int l8, in
   }
   // Divisions.  x / b as q0 = x*r, rem = fma(-q0, b, x), q = fma(rem, r, q0) with r = RN(1/b) is the correctly
   // rounded quotient for every divisor used here (3, 15 and the 126 positive E4M3 values: checked against
-  // IEEE division for all 2^23 significands of x), as long as nothing over- or underflows; operands outside
-  // [2^-60, 2^60] (other than 0) take the IEEE division instead, the whole warp together.
+  // IEEE division for all 2^23 significands of x) as long as nothing overflows.  A quotient too small to be
+  // computed exactly needs no care: it is below 2^-40 and rounds to the integer 0, or to the step floor 2^-9,
+  // either way.  Rounding to an integer is q + 1.5*2^23 - 1.5*2^23 (the FMA pipe instead of the quarter-rate
+  // conversion unit), which is rint(q) while |q| < 2^22.  Vectors with magnitudes or quotients beyond those
+  // bounds take IEEE division and rintf instead, the whole warp together.
   const float range = __fsub_rn(mx, mn);
-  float amax = fmaxf(fabsf(range), fmaxf(fabsf(mn), fabsf(mx)));
-  float amin = fabsf(range) > 0.f ? fabsf(range) : 1.f;
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) amin = fminf(amin, x[e] != 0.f ? fabsf(x[e]) : 1.f);
-  amin = fminf(amin, mn != 0.f ? fabsf(mn) : 1.f);
-  const bool slow = __any_sync(0xFFFFFFFFu, !(amax < 0x1p60f) || !(amin > 0x1p-60f));
+  const float amax = fmaxf(fabsf(range), fmaxf(fabsf(mn), fabsf(mx)));
   auto fast_div = [](float a, float b, float r) {
     const float q0 = __fmul_rn(a, r);
     return __fmaf_rn(__fmaf_rn(-q0, b, a), r, q0);
   };
-  const float step = slow ? __fdiv_rn(range, L) : fast_div(range, L, (BITS == 2) ? __uint_as_float(0x3EAAAAABu) : __uint_as_float(0x3D888889u));
+  const bool big = !(amax < 0x1p60f);
+  float step = fast_div(range, L, (BITS == 2) ? __uint_as_float(0x3EAAAAABu) : __uint_as_float(0x3D888889u));
+  if (big) step = __fdiv_rn(range, L);
   uint32_t sbyte = f32_to_e4m3_byte(step);
   if (sbyte == 0) sbyte = 1;                       // floor at the smallest subnormal 2^-9
   const float ds = e4m3_byte_to_f32(sbyte);
   const float rds = __frcp_rn(ds);
-  const float z = __fsub_rn(0.0f, rintf(slow ? __fdiv_rn(mn, ds) : fast_div(mn, ds, rds)));
+  const bool slow = __any_sync(0xFFFFFFFFu, big || !(__fmul_rn(amax, rds) < 0x1p21f));
+  constexpr float kRound = 12582912.f;             // 1.5 * 2^23
+  const float z = __fsub_rn(0.0f, slow ? rintf(__fdiv_rn(mn, ds)) : __fsub_rn(__fadd_rn(fast_div(mn, ds, rds), kRound), kRound));
   const uint32_t zbits = f32_to_bf16_bits(z);
   const float zs = bf16_bits_to_f32(zbits);
 
-  uint32_t piece[(kBitsPerLane + 31) / 32] = {};
+  // Codes are packed 16 bits at a time as exact float sums c_e * 2^(bit position), then read out of the low
+  // mantissa bits of sum + 2^23.
+  constexpr int kChunks = kBitsPerLane / 16;
+  float acc[kChunks];
+#pragma unroll
+  for (int k = 0; k < kChunks; ++k) acc[k] = 8388608.f;
   if (!slow) {
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
-      float c = __fadd_rn(rintf(fast_div(x[e], ds, rds)), zs);
-      c = fminf(fmaxf(c, 0.0f), L);
-      // c is an integer in [0, L]: adding 2^23 leaves it in the low mantissa bits
-      piece[(e * BITS) / 32] |= (__float_as_uint(__fadd_rn(c, 8388608.f)) & (uint32_t)L) << ((e * BITS) % 32);
+      const float r = __fsub_rn(__fadd_rn(fast_div(x[e], ds, rds), kRound), kRound);
+      const float c = fminf(fmaxf(__fadd_rn(r, zs), 0.0f), L);
+      acc[(e * BITS) / 16] = __fmaf_rn(c, (float)(1u << ((e * BITS) % 16)), acc[(e * BITS) / 16]);
     }
   } else {
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
-      float c = __fadd_rn(rintf(__fdiv_rn(x[e], ds)), zs);
-      c = fminf(fmaxf(c, 0.0f), L);
-      piece[(e * BITS) / 32] |= ((uint32_t)c) << ((e * BITS) % 32);
+      const float c = fminf(fmaxf(__fadd_rn(rintf(__fdiv_rn(x[e], ds)), zs), 0.0f), L);
+      acc[(e * BITS) / 16] = __fmaf_rn(c, (float)(1u << ((e * BITS) % 16)), acc[(e * BITS) / 16]);
     }
+  }
+  uint32_t piece[(kBitsPerLane + 31) / 32];
+  if constexpr (kChunks == 1) {
+    piece[0] = __float_as_uint(acc[0]) & 0xFFFFu;
+  } else {
+#pragma unroll
+    for (int k = 0; k < kChunks; k += 2)
+      piece[k / 2] = __byte_perm(__float_as_uint(acc[k]), __float_as_uint(acc[k + 1]), 0x5410);
   }
   if constexpr (kBitsPerLane == 16) {                  // two lanes share a word
     const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, piece[0], 1);

@@ -93,6 +93,11 @@ def test_degenerate_groups_and_strided_input(B):
     x[0, 1, 3] *= 1e4                   # step saturates E4M3 (448)
     x[0, 1, 4] *= 1e-6                  # step in the subnormal range / floored
     x[0, 1, 5] += 100.0                 # large zero-point
+    x[0, 1, 6] *= 1e25                  # magnitudes beyond 2^60: the kernel's IEEE-division path
+    x[0, 1, 7] *= 1e-25                 # magnitudes far below the step floor
+    x[0, 1, 8, ::3] *= 1e-30            # tiny elements inside a normal range
+    x[0, 1, 9] = 1e6 + 1e-3 * x[0, 1, 9]   # quotients x/step beyond 2^21 (zero-point far outside BF16's integers)
+    x[0, 1, 10, :32] = 3e4              # a constant group whose quotient is large
     kb = inputs.f32_to_bf16_bits(x)
     vb = inputs.f32_to_bf16_bits(x[..., ::-1].copy())
     for rotate in (False, True):
