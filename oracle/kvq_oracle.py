@@ -209,6 +209,18 @@ class Cache:
     capacity: int
     rotate_k: bool = True
     signs: np.ndarray | None = None
+    ring: bool = False      # sliding-window use (Sec. 2: attend to the last n cached chunks): token t lives in slot t mod capacity
+
+    def slots(self, begin, n):
+        """Slots of the tokens [begin, begin + n): themselves, or taken modulo the capacity for a ring cache."""
+        idx = np.arange(begin, begin + n, dtype=np.int64)
+        if self.ring:
+            if n > self.capacity:
+                raise ValueError("more tokens than slots")
+            return idx % self.capacity
+        if begin + n > self.capacity:
+            raise ValueError("capacity exceeded")
+        return idx
 
     def __post_init__(self):
         B, H, C, d = self.batch, self.heads, self.capacity, self.head_dim
@@ -228,17 +240,16 @@ class Cache:
 
 def quantize_append(cache: Cache, cache_len: int, k_bits, v_bits):
     """Rotate (keys only), quantize, pack and store a finished chunk at tokens
-    [cache_len, cache_len + n).  k_bits, v_bits: BF16 bit patterns [B, H, n, d]."""
+    [cache_len, cache_len + n) (slots taken modulo the capacity for a ring cache, where the
+    new tokens overwrite the oldest ones).  k_bits, v_bits: BF16 bit patterns [B, H, n, d]."""
     n = k_bits.shape[2]
-    if cache_len + n > cache.capacity:
-        raise ValueError("capacity exceeded")
+    sl = cache.slots(cache_len, n)
     k = bf16_bits_to_f64(k_bits)
     v = bf16_bits_to_f64(v_bits)
     if cache.rotate_k:
         k = rotate_f32_steps(k, cache.signs)
     kc, ks, kz = quantize_vectors(k, cache.bits, cache.group)
     vc, vs, vz = quantize_vectors(v, cache.bits, cache.group)
-    sl = slice(cache_len, cache_len + n)
     cache.k_codes[:, :, sl] = pack_codes(kc, cache.bits)
     cache.v_codes[:, :, sl] = pack_codes(vc, cache.bits)
     cache.k_scale[:, :, sl] = ks
@@ -338,7 +349,7 @@ def attn_corrected(cache: Cache, cache_begin, cache_len, q_bits, kcur_bits, vcur
     Returns dict of arrays indexed [unit, row, ...] in the order of `heads`."""
     B, H = q_bits.shape[:2]
     units = heads if heads is not None else [(b, h) for b in range(B) for h in range(H)]
-    sl = slice(cache_begin, cache_begin + cache_len)
+    sl = cache.slots(cache_begin, cache_len)
     outs, lses, masses, cmasses = [], [], [], []
     for (b, h) in units:
         r = attn_corrected_head(

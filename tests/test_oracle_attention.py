@@ -201,6 +201,40 @@ def test_window_and_row_subset():
     assert np.array_equal(win["out"], O.attn_corrected(c2, 0, 16, q, kc, vc, 0.125)["out"])
 
 
+def test_ring_cache_is_the_sliding_window():
+    """A ring cache of C slots after appending T > C tokens, attended over its last W tokens, must give exactly
+    what a linear cache holding all T tokens gives over the same window [T - W, T): the ring only changes where
+    a token is stored (slot t mod C), and the newest tokens overwrite the oldest."""
+    d, bits, group, C = 64, 2, 32, 48
+    w = inputs.Workload("ring", 77, 1, 2, d, 20, 0, bits, group, 5)
+    ring = O.Cache(1, 2, d, bits, group, C, ring=True)
+    lin = O.Cache(1, 2, d, bits, group, 200)
+    n = 0
+    for c in range(7):                                   # 140 tokens through 48 slots: wraps twice, chunks straddle the end
+        _, k, v = inputs.make_chunk(w, c)
+        assert O.quantize_append(ring, n, k, v) == O.quantize_append(lin, n, k, v)
+        n += 20
+    q, kc, vc = inputs.make_chunk(w, 9)
+    for W in (48, 40, 13, 0):
+        a = O.attn_corrected(ring, n - W, W, q, kc, vc, 0.125)
+        b = O.attn_corrected(lin, n - W, W, q, kc, vc, 0.125)
+        for key in ("out", "lse", "cached_mass"):
+            assert np.array_equal(a[key], b[key]), (W, key)
+    # slot s holds the newest token t with t = s (mod C), by brute force over the stored bytes
+    for s_ in range(C):
+        t = max(t for t in range(n) if t % C == s_)
+        assert np.array_equal(ring.k_codes[:, :, s_], lin.k_codes[:, :, t])
+        assert np.array_equal(ring.v_zero[:, :, s_], lin.v_zero[:, :, t])
+    # a window longer than the ring, or a linear cache run past its end, is refused
+    for bad in (lambda: O.attn_corrected(ring, n - 49, 49, q, kc, vc, 0.125),
+                lambda: O.quantize_append(lin, 190, *inputs.make_chunk(w, 0)[1:])):
+        try:
+            bad()
+            raise AssertionError("accepted")
+        except ValueError:
+            pass
+
+
 def _brute_force(q_bits, kc_bits, vc_bits, cache, n_s, sigma, correction):
     """Algorithm 1 with Python loops, its own dequantization from the stored bytes and
     an explicit Hadamard matrix.  Written separately from the oracle."""
