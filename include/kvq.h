@@ -56,6 +56,12 @@ extern "C" {
 
 /* kvq_cache_desc.flags */
 #define KVQ_ROTATE_K          1u   /* keys (and queries) are Hadamard-rotated before quantization */
+#define KVQ_RING              2u   /* ring cache for sliding-window attention (Section 2; the windows of Section 5.1):
+                                      token t lives in slot t mod capacity, new tokens overwrite the oldest.  Token
+                                      positions (cache_len of kvq_quantize_append, cache_begin of the attention calls)
+                                      are then unbounded; one append may bring at most `capacity` tokens and a window
+                                      may hold at most `capacity` tokens.  Which tokens are still stored is the
+                                      caller's bookkeeping: the last `capacity` appended ones. */
 
 /* kvq_attn_corrected flags */
 #define KVQ_CORRECTION_OFF    0u
@@ -72,7 +78,7 @@ typedef struct kvq_cache_desc {
   int32_t  batch, heads, head_dim;   /* head_dim: 64 or 128 */
   int32_t  bits;                     /* 2 or 4 */
   int32_t  group;                    /* 32, 64 or 128; divides head_dim */
-  uint32_t flags;                    /* KVQ_ROTATE_K */
+  uint32_t flags;                    /* KVQ_ROTATE_K | KVQ_RING */
   int64_t  capacity;                 /* tokens per (batch, head); a multiple of 128 */
   void*    k_codes;  void* v_codes;  /* device, u8  [batch,heads,capacity, head_dim*bits/8] */
   void*    k_scale;  void* v_scale;  /* device, u8  [batch,heads,capacity, head_dim/group] (E4M3) */

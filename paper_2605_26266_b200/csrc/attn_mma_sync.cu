@@ -281,12 +281,16 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
   // ---- cached segment ----------------------------------------------------------------
   const int key = tid >> 1, half = tid & 1;
   const int n_ctiles = (p.n_cached + kBN - 1) / kBN;
-  const int64_t tok_base = (int64_t)bh * p.capacity + p.cache_begin;
+  const int64_t tok_base = (int64_t)bh * p.capacity;
   if (n_ctiles > 0) {
     load_q_frags(sQr);
     Packed<D, BITS> pk, pv;
     // reading past n_cached stays inside `capacity` only up to the last token; clamp the index
-    auto tok_of = [&](int t) { return tok_base + min((int64_t)t * kBN + key, (int64_t)p.n_cached - 1); };
+    // window key -> slot, modulo the capacity (ring caches wrap)
+    auto tok_of = [&](int t) {
+      const int64_t slot = p.cache_begin + min((int64_t)t * kBN + key, (int64_t)p.n_cached - 1);
+      return tok_base + (slot >= p.capacity ? slot - p.capacity : slot);
+    };
     load_packed<D, BITS>(pk, p.k_codes, p.k_scale, p.k_zero, tok_of(0), half, G);
     load_packed<D, BITS>(pv, p.v_codes, p.v_scale, p.v_zero, tok_of(0), half, G);
     for (int t = 0; t < n_ctiles; ++t) {
@@ -392,7 +396,7 @@ int launch_attn_mma_sync(const AttnArgs& a) {
   p.k_scale = static_cast<const uint8_t*>(d->k_scale); p.v_scale = static_cast<const uint8_t*>(d->v_scale);
   p.k_zero = static_cast<const uint16_t*>(d->k_zero); p.v_zero = static_cast<const uint16_t*>(d->v_zero);
   p.signs = d->signs;
-  p.capacity = d->capacity; p.cache_begin = a.cache_begin;
+  p.capacity = d->capacity; p.cache_begin = a.cache_begin % d->capacity;
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
   p.correction = (a.flags & KVQ_CORRECTION_ON) ? 1 : 0;
   p.m_tokens = (int)a.m_tokens; p.n_cached = (int)a.cache_len; p.n_cur = (int)a.n_cur;

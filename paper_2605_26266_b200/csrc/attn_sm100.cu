@@ -856,12 +856,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     Raw<BITS> rk, rv;
     while (ok && sch.next(sg)) {
       const int bh = sg.unit / p.q_blocks;
-      const int64_t tok0 = (int64_t)bh * p.capacity + p.cache_begin;
+      // key k of the window lives in slot cache_begin + k, taken modulo the capacity (ring caches wrap; for
+      // linear ones the host has checked that the window ends inside the capacity)
+      const int64_t slab0 = (int64_t)bh * p.capacity;
+      auto tok_of = [&](int k) {
+        const int64_t slot = p.cache_begin + k;
+        return slab0 + (slot >= p.capacity ? slot - p.capacity : slot);
+      };
       const int t_rot = max(sg.tb, n_rt);          // first cached tile of the segment: the query is rotated there
       if (sg.te > n_rt) {
         const int k0 = (t_rot - n_rt) * kBlockN + dt;
-        load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k0, k0 < p.n_cached);
-        load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k0, k0 < p.n_cached);
+        load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k0), k0 < p.n_cached);
+        load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(k0), k0 < p.n_cached);
       }
       for (int t = sg.tb; t < sg.te; ++t, ++it) {
         const int s = it & 1;
@@ -879,7 +885,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(dt, 0)) = make_uint4(b01, b23, b01, b23);
           }
           fence_proxy_async_smem();
-          if (t + 1 < sg.te) load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok0 + k1, k1 < p.n_cached);
+          if (t + 1 < sg.te) load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k1), k1 < p.n_cached);
         }
         mbar_arrive(cx.bar(kKFull + s));
         if (t == t_rot) {
@@ -903,7 +909,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (ct >= 0) {
           dequant_values<BITS, GROUP>(rv, smem + kOffV + s * kTileBytes, dt);
           fence_proxy_async_smem();
-          if (t + 1 < sg.te) load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok0 + k1, k1 < p.n_cached);
+          if (t + 1 < sg.te) load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(k1), k1 < p.n_cached);
         }
         mbar_arrive(cx.bar(kVFull + s));
       }
@@ -1151,7 +1157,7 @@ static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t
   p.k_scale = static_cast<const uint8_t*>(d->k_scale); p.v_scale = static_cast<const uint8_t*>(d->v_scale);
   p.k_zero = static_cast<const uint16_t*>(d->k_zero); p.v_zero = static_cast<const uint16_t*>(d->v_zero);
   p.signs = d->signs;
-  p.capacity = d->capacity; p.cache_begin = a.cache_begin;
+  p.capacity = d->capacity; p.cache_begin = a.cache_begin % d->capacity;
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
   p.correction = (a.flags & KVQ_CORRECTION_ON) ? 1 : 0;
   p.m_tokens = (int)a.m_tokens; p.n_cached = (int)a.cache_len; p.n_cur = (int)a.n_cur;

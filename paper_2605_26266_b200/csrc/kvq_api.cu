@@ -19,6 +19,7 @@ int check_shape(const kvq_cache_desc* d) {
   if (d->bits != 2 && d->bits != 4) return KVQ_ERR_UNSUPPORTED;
   if (d->group != 32 && d->group != 64 && d->group != 128) return KVQ_ERR_UNSUPPORTED;
   if (d->capacity % 128 != 0) return KVQ_ERR_INVALID_ARG;
+  if (d->flags & ~(KVQ_ROTATE_K | KVQ_RING)) return KVQ_ERR_INVALID_ARG;
   return KVQ_OK;
 }
 
@@ -47,7 +48,8 @@ static int check_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t
   if (r != KVQ_OK) return r;
   if (cache_begin < 0 || cache_len < 0 || m_tokens < 0 || n_cur < 1) return KVQ_ERR_INVALID_ARG;
   if (cache_begin % 16 != 0) return KVQ_ERR_ALIGNMENT;
-  if (cache_begin + cache_len > d->capacity) return KVQ_ERR_CAPACITY;
+  // linear cache: the window ends inside the capacity; ring cache: it has at most `capacity` tokens
+  if (((d->flags & KVQ_RING) ? cache_len : cache_begin + cache_len) > d->capacity) return KVQ_ERR_CAPACITY;
   if (m_tokens > 0x7FFFFFFFLL || n_cur > 0x7FFFFFFFLL || cache_len > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
   const uint32_t kern = flags & KVQ_KERNEL_MASK;
   if (kern != KVQ_KERNEL_AUTO && kern != KVQ_KERNEL_MMA_SYNC && kern != KVQ_KERNEL_TCGEN05)
@@ -106,7 +108,7 @@ int kvq_quantize_append(const kvq_cache_desc* desc, int64_t cache_len, const voi
   int r = check_desc(desc);
   if (r != KVQ_OK) return r;
   if (cache_len < 0 || n_tokens < 0) return KVQ_ERR_INVALID_ARG;
-  if (cache_len + n_tokens > desc->capacity) return KVQ_ERR_CAPACITY;
+  if (((desc->flags & KVQ_RING) ? n_tokens : cache_len + n_tokens) > desc->capacity) return KVQ_ERR_CAPACITY;
   if ((r = check_tensor(k_bf16, kv)) != KVQ_OK) return r;
   if ((r = check_tensor(v_bf16, kv)) != KVQ_OK) return r;
   if (n_tokens == 0) return KVQ_OK;
@@ -203,7 +205,7 @@ int kvq_unpack_codes(const kvq_cache_desc* desc, int which, int64_t begin, int64
   int r = check_desc(desc);
   if (r != KVQ_OK) return r;
   if ((which != 0 && which != 1) || begin < 0 || n < 0 || !out_codes) return KVQ_ERR_INVALID_ARG;
-  if (begin + n > desc->capacity) return KVQ_ERR_CAPACITY;
+  if (((desc->flags & KVQ_RING) ? n : begin + n) > desc->capacity) return KVQ_ERR_CAPACITY;
   return launch_unpack_codes(desc, which, begin, n, out_codes, (cudaStream_t)stream);
 }
 

@@ -149,7 +149,7 @@ __device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int l8, in
 
 // Cooperative shared->global copy with the widest store both sides allow.
 __device__ __forceinline__ void copy_out(uint8_t* dst, const uint8_t* src, int nbytes, int tid, int nthreads) {
-  const uintptr_t a = reinterpret_cast<uintptr_t>(dst) | (uintptr_t)nbytes;
+  const uintptr_t a = reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src) | (uintptr_t)nbytes;
   if ((a & 15) == 0) {
     for (int i = tid; i < nbytes / 16; i += nthreads)
       reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
@@ -241,13 +241,24 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
     decode_vec<EPL>(rv_cur, x);
     quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[1], s_scale[1], s_zero[1]);
     __syncthreads();
-    const int64_t tok_index = (int64_t)bh * p.capacity + p.cache_len + t0;
+    // The tile goes to slots slot0 .. slot0 + nt - 1, modulo the capacity: one piece, or two when a ring
+    // cache wraps inside the tile (p.cache_len is already reduced modulo the capacity, so one subtraction does).
+    int64_t slot0 = p.cache_len + t0;
+    if (slot0 >= p.capacity) slot0 -= p.capacity;
+    const int n_first = (int)min((int64_t)nt, p.capacity - slot0);
+#pragma unroll 1
+    for (int piece = 0; piece < 2; ++piece) {
+      const int ntok = piece ? nt - n_first : n_first;
+      if (ntok <= 0) break;
+      const int skip = piece ? n_first : 0;                    // tokens of the tile stored by the first piece
+      const int64_t tok_index = (int64_t)bh * p.capacity + (piece ? 0 : slot0);
 #pragma unroll
-    for (int w = 0; w < 2; ++w) {
-      copy_out(p.codes[w] + tok_index * CB, reinterpret_cast<const uint8_t*>(s_codes[w]), nt * CB, threadIdx.x, kWarps * 32);
-      copy_out(p.scale[w] + tok_index * G, s_scale[w], nt * G, threadIdx.x, kWarps * 32);
-      copy_out(reinterpret_cast<uint8_t*>(p.zero[w] + tok_index * G), reinterpret_cast<const uint8_t*>(s_zero[w]),
-               nt * G * 2, threadIdx.x, kWarps * 32);
+      for (int w = 0; w < 2; ++w) {
+        copy_out(p.codes[w] + tok_index * CB, reinterpret_cast<const uint8_t*>(s_codes[w]) + skip * CB, ntok * CB, threadIdx.x, kWarps * 32);
+        copy_out(p.scale[w] + tok_index * G, s_scale[w] + skip * G, ntok * G, threadIdx.x, kWarps * 32);
+        copy_out(reinterpret_cast<uint8_t*>(p.zero[w] + tok_index * G), reinterpret_cast<const uint8_t*>(s_zero[w] + skip * G),
+                 ntok * G * 2, threadIdx.x, kWarps * 32);
+      }
     }
     __syncthreads();
   }
@@ -262,7 +273,9 @@ __global__ void unpack_codes_kernel(const uint8_t* codes, uint8_t* out, int64_t 
   const int64_t t = (i / D) % n;
   const int64_t bh = i / ((int64_t)D * n);
   const int CB = D * BITS / 8;
-  const uint8_t byte = codes[(bh * capacity + begin + t) * CB + (c * BITS) / 8];
+  int64_t slot = begin + t;                                   // begin is already reduced modulo the capacity
+  if (slot >= capacity) slot -= capacity;
+  const uint8_t byte = codes[(bh * capacity + slot) * CB + (c * BITS) / 8];
   out[i] = (byte >> ((c * BITS) % 8)) & ((1 << BITS) - 1);
 }
 
@@ -274,7 +287,7 @@ int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const voi
   p.k = static_cast<const uint16_t*>(k);
   p.v = static_cast<const uint16_t*>(v);
   p.sb = kv.b; p.sh = kv.h; p.st = kv.t;
-  p.n_tokens = n_tokens; p.cache_len = cache_len; p.capacity = d->capacity;
+  p.n_tokens = n_tokens; p.cache_len = cache_len % d->capacity; p.capacity = d->capacity;
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
   p.signs = d->signs;
   p.codes[0] = static_cast<uint8_t*>(d->k_codes); p.codes[1] = static_cast<uint8_t*>(d->v_codes);
@@ -310,9 +323,9 @@ int launch_unpack_codes(const kvq_cache_desc* d, int which, int64_t begin, int64
   const int64_t blocks = (total + threads - 1) / threads;
   if (blocks > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
   if (d->bits == 2)
-    unpack_codes_kernel<2><<<(unsigned)blocks, threads, 0, st>>>(codes, out, d->capacity, begin, n, d->head_dim, total);
+    unpack_codes_kernel<2><<<(unsigned)blocks, threads, 0, st>>>(codes, out, d->capacity, begin % d->capacity, n, d->head_dim, total);
   else
-    unpack_codes_kernel<4><<<(unsigned)blocks, threads, 0, st>>>(codes, out, d->capacity, begin, n, d->head_dim, total);
+    unpack_codes_kernel<4><<<(unsigned)blocks, threads, 0, st>>>(codes, out, d->capacity, begin % d->capacity, n, d->head_dim, total);
   KVQ_CUDA_TRY(cudaGetLastError());
   return KVQ_OK;
 }

@@ -81,3 +81,24 @@ def test_argument_errors_without_gpu(binding):
     assert args(0, 16, 0, 16, 1 | b.KVQ_KERNEL_MMA_SYNC) == b.KVQ_OK                             # m = 0: no-op
     assert b.lib.kvq_unpack_codes(C.byref(ok), 2, 0, 4, 0x1000, None) == b.KVQ_ERR_INVALID_ARG
     assert b.lib.kvq_unpack_codes(C.byref(ok), 0, 250, 16, 0x1000, None) == b.KVQ_ERR_CAPACITY
+
+
+def test_ring_cache_argument_rules_without_gpu(binding):
+    b = binding
+    ring = b.kvq_cache_desc(1, 2, 128, 2, 32, b.KVQ_ROTATE_K | b.KVQ_RING, 256)
+    for f in ("k_codes", "v_codes", "k_scale", "v_scale", "k_zero", "v_zero"):
+        setattr(ring, f, 0x10000)
+    s = b.kvq_strides(2 * 256 * 128, 256 * 128, 128)
+    # positions are unbounded, but one append and one window hold at most `capacity` tokens
+    assert b.lib.kvq_quantize_append(C.byref(ring), 10 ** 9, 0x1000, 0x1000, s, 0, None) == b.KVQ_OK
+    assert b.lib.kvq_quantize_append(C.byref(ring), 250, 0x1000, 0x1000, s, 257, None) == b.KVQ_ERR_CAPACITY
+    args = lambda begin, n_cache, m: b.lib.kvq_attn_corrected(
+        C.byref(ring), begin, n_cache, 0x1000, s, 0x1000, 0x1000, s, m, 16, 0x1000, s, 0.088, 1,
+        None, None, None, 0, None, None)
+    assert args(1024, 256, 0) == b.KVQ_OK            # m = 0: checks only
+    assert args(1024, 257, 0) == b.KVQ_ERR_CAPACITY
+    assert args(1000, 16, 0) == b.KVQ_ERR_ALIGNMENT
+    assert b.lib.kvq_unpack_codes(C.byref(ring), 0, 250, 257, 0x1000, None) == b.KVQ_ERR_CAPACITY
+    unknown = b.kvq_cache_desc(1, 2, 128, 2, 32, 4, 256)
+    sizes = (C.c_size_t * 6)()
+    assert b.lib.kvq_cache_bytes(C.byref(unknown), sizes) == b.KVQ_ERR_INVALID_ARG
