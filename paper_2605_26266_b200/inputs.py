@@ -84,6 +84,8 @@ WORKLOADS = {
     "long": Workload("long", 4, 1, 24, 128, 4680, 32, 2, 128, 0),
     "pipeline": Workload("pipeline", 5, 2, 32, 128, 2048, 15, 2, 32, 1,
                          k_dist="student_t3", k_outliers=8, k_outlier_scale=10.0),
+    # short query chunk over a long prefix (the partial-prefill regime): 32 units of 514 key tiles, split over all SMs
+    "prefix": Workload("prefix", 6, 1, 32, 128, 256, 256, 2, 128, 0, k_outliers=4, k_outlier_scale=8.0),
 }
 
 

@@ -206,7 +206,7 @@ def test_sweep_config_full_rows(B, name, seed):
     _compare(B, g, o, n, q, kc, vc, T.sigma_of(w.head_dim), sel)
 
 
-@pytest.mark.parametrize("name,units", [("dit", [(0, 2), (0, 23)]), ("long", [(0, 13)])])
+@pytest.mark.parametrize("name,units", [("dit", [(0, 2), (0, 23)]), ("long", [(0, 13)]), ("prefix", [(0, 5), (0, 31)])])
 def test_large_configs_sampled_rows(B, name, units):
     """Full-size launch; oracle on sampled rows touching every 128-row tile, for a few heads."""
     w = inputs.WORKLOADS[name]
