@@ -65,7 +65,12 @@ extern "C" {
 
 /* kvq_attn_corrected flags */
 #define KVQ_CORRECTION_OFF    0u
-#define KVQ_CORRECTION_ON     1u   /* subtract the Taylor bias from cached scores */
+#define KVQ_CORRECTION_ON     1u   /* subtract the Taylor bias (Eq. 15 / Eq. 25) from cached scores */
+#define KVQ_CORRECTION_EXACT  2u   /* subtract the exact bias of Eq. (12) instead: sum over channels of
+                                      log(sinh(a)/a), a = softmax_scale * |q~_c| * step / 2.  Not together with
+                                      KVQ_CORRECTION_ON.  Warp-level kernel only (KVQ_KERNEL_AUTO picks it;
+                                      KVQ_KERNEL_TCGEN05 and the static-scratch entry return
+                                      KVQ_ERR_UNSUPPORTED): an analysis option, several times slower. */
 #define KVQ_KERNEL_AUTO       0u
 #define KVQ_KERNEL_MMA_SYNC   (1u << 8)  /* force the warp-level mma.sync kernel (cross-check / fallback shapes) */
 #define KVQ_KERNEL_TCGEN05    (2u << 8)  /* force the tcgen05/TMEM kernel; KVQ_ERR_UNSUPPORTED if the shape is not covered */

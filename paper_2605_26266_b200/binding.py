@@ -21,7 +21,7 @@ KVQ_ERR_INVALID_ARG, KVQ_ERR_UNSUPPORTED, KVQ_ERR_ALIGNMENT = -1, -2, -3
 KVQ_ERR_CAPACITY, KVQ_ERR_CUDA, KVQ_ERR_TIMEOUT, KVQ_ERR_WORKSPACE = -4, -5, -6, -7
 KVQ_ROTATE_K = 1
 KVQ_RING = 2
-KVQ_CORRECTION_OFF, KVQ_CORRECTION_ON = 0, 1
+KVQ_CORRECTION_OFF, KVQ_CORRECTION_ON, KVQ_CORRECTION_EXACT = 0, 1, 2
 KVQ_KERNEL_AUTO, KVQ_KERNEL_MMA_SYNC, KVQ_KERNEL_TCGEN05 = 0, 1 << 8, 2 << 8
 
 

@@ -29,9 +29,10 @@ struct AParams {
   const uint16_t* k_zero; const uint16_t* v_zero;
   const int8_t* signs;
   int64_t capacity, cache_begin;
-  int heads, group, rotate, correction;
+  int heads, group, rotate, correction;   // correction: 0 off, 1 Taylor (Eq. 15), 2 exact (Eq. 12)
   int m_tokens, n_cached, n_cur;
   float scale_log2, bias_coef_log2;   // sigma*log2(e), (sigma^2/24)*log2(e)
+  float softmax_scale;
   float* lse; float* cached_mass;
 };
 
@@ -112,6 +113,15 @@ __device__ __forceinline__ void dequant_store(const Packed<D, BITS>& r, uint16_t
   }
 }
 
+// log(sinh(a)/a) for a >= 0 (Eq. (12)): series below 0.5, a - log(2a) + log1p(-exp(-2a)) above.
+__device__ __forceinline__ float log_sinhc(float a) {
+  if (a < 0.5f) {
+    const float a2 = a * a;
+    return a2 * (1.0f / 6.0f + a2 * (-1.0f / 180.0f + a2 * (1.0f / 2835.0f - a2 * (1.0f / 37800.0f))));
+  }
+  return a - __logf(2.0f * a) + log1pf(-__expf(-2.0f * a));
+}
+
 template <int D, int BITS>
 __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
   constexpr int LD = D + 8;
@@ -125,6 +135,11 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
   uint16_t* sV = sK + kBN * LD;                                // value tile       [kBN][LD]
   float* sNu = reinterpret_cast<float*>(sV + kBN * LD);        // [kBM][4]
   float* sW = sNu + kBM * 4;                                   // [kBN][4]
+  // exact correction only: E4M3 step bytes of the tile's keys, and per (row, group, step byte) the bias
+  // log2(e) * sum over the group's channels of log(sinh(a)/a), a = sigma |q~_c| step / 2 (Eq. (12)): a step
+  // takes one of 127 values, so the exact bias of a score is one table look-up per group
+  uint32_t* sWb = reinterpret_cast<uint32_t*>(sW + kBN * 4);   // [kBN]
+  float* sT = reinterpret_cast<float*>(sWb + kBN);             // [kBM][G][128]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.y, b = bh / p.heads, h = bh - b * p.heads;
@@ -177,6 +192,17 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
       for (int e = 0; e < EPL; ++e) nu += x[e] * x[e];
       for (int off = 1; off < lanes_per_group; off *= 2) nu += __shfl_xor_sync(0xFFFFFFFFu, nu, off);
       if ((lane % lanes_per_group) == 0) sNu[r * 4 + lane / lanes_per_group] = nu;
+      if (p.correction == 2) {
+        const int j = lane / lanes_per_group;
+        for (int e = 0; e < 128; ++e) {
+          const float half_step = 0.5f * p.softmax_scale * e4m3_byte_to_f32((uint32_t)e);
+          float t = 0.f;
+#pragma unroll
+          for (int c = 0; c < EPL; ++c) t += log_sinhc(fabsf(x[c]) * half_step);
+          for (int off = 1; off < lanes_per_group; off *= 2) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
+          if ((lane % lanes_per_group) == 0) sT[(r * G + j) * 128 + e] = (e == 127) ? 0.f : t * kLog2e;
+        }
+      }
 #pragma unroll
       for (int e = 0; e < EPL / 2; ++e)
         reinterpret_cast<uint32_t*>(sQr + r * LD + lane * EPL)[e] = pack_f16(x[2 * e], x[2 * e + 1]);
@@ -229,10 +255,17 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
         const int col = nb * 8 + (lane & 3) * 2 + (e & 1);
         float v = s[nb][e] * p.scale_log2;
         if (biased) {
-          const float* nu = (e < 2) ? nuA : nuB;
           float bsum = 0.f;
+          if (p.correction == 2) {
+            const float* trow = sT + (size_t)((e < 2) ? rA : rB) * G * 128;
+            const uint32_t sb = sWb[col];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) bsum += (j < G) ? nu[j] * sW[col * 4 + j] : 0.f;
+            for (int j = 0; j < 4; ++j) bsum += (j < G) ? trow[j * 128 + ((sb >> (8 * j)) & 0x7Fu)] : 0.f;
+          } else {
+            const float* nu = (e < 2) ? nuA : nuB;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bsum += (j < G) ? nu[j] * sW[col * 4 + j] : 0.f;
+          }
           v -= bsum;
         }
         if (col >= n_valid) v = -INFINITY;
@@ -303,6 +336,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
           const float ds = e4m3_byte_to_f32((pk.sbytes >> (8 * j)) & 0xFFu);
           sW[key * 4 + j] = (p.correction && j < G) ? p.bias_coef_log2 * ds * ds : 0.f;
         }
+        sWb[key] = pk.sbytes;
       }
       __syncthreads();
       if (t + 1 < n_ctiles) {
@@ -371,10 +405,13 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
 template <int D, int BITS>
 int launch(const AParams& p, dim3 grid, cudaStream_t st) {
   constexpr int LD = D + 8;
-  constexpr size_t smem = (size_t)(2 * kBM + 2 * kBN) * LD * 2 + (kBM + kBN) * 4 * sizeof(float);
+  constexpr size_t base = (size_t)(2 * kBM + 2 * kBN) * LD * 2 + (kBM + kBN) * 4 * sizeof(float) + kBN * sizeof(uint32_t);
+  // the exact correction adds its table: 64 rows x groups x 128 step values
+  const size_t smem = base + (p.correction == 2 ? (size_t)kBM * (D / p.group) * 128 * sizeof(float) : 0);
   static bool configured = false;
   if (!configured) {
-    KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_mma_sync_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_mma_sync_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)(base + (size_t)kBM * 4 * 128 * sizeof(float))));
     configured = true;
   }
   attn_mma_sync_kernel<D, BITS><<<grid, kThreads, smem, st>>>(p);
@@ -398,7 +435,8 @@ int launch_attn_mma_sync(const AttnArgs& a) {
   p.signs = d->signs;
   p.capacity = d->capacity; p.cache_begin = a.cache_begin % d->capacity;
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
-  p.correction = (a.flags & KVQ_CORRECTION_ON) ? 1 : 0;
+  p.correction = (a.flags & KVQ_CORRECTION_EXACT) ? 2 : ((a.flags & KVQ_CORRECTION_ON) ? 1 : 0);
+  p.softmax_scale = a.softmax_scale;
   p.m_tokens = (int)a.m_tokens; p.n_cached = (int)a.cache_len; p.n_cur = (int)a.n_cur;
   p.scale_log2 = a.softmax_scale * kLog2e;
   p.bias_coef_log2 = a.softmax_scale * a.softmax_scale / 24.0f * kLog2e;

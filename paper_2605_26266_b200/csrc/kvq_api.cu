@@ -54,7 +54,8 @@ static int check_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t
   const uint32_t kern = flags & KVQ_KERNEL_MASK;
   if (kern != KVQ_KERNEL_AUTO && kern != KVQ_KERNEL_MMA_SYNC && kern != KVQ_KERNEL_TCGEN05)
     return KVQ_ERR_INVALID_ARG;
-  if (flags & ~(KVQ_CORRECTION_ON | KVQ_KERNEL_MASK)) return KVQ_ERR_INVALID_ARG;
+  if (flags & ~(KVQ_CORRECTION_ON | KVQ_CORRECTION_EXACT | KVQ_KERNEL_MASK)) return KVQ_ERR_INVALID_ARG;
+  if ((flags & KVQ_CORRECTION_ON) && (flags & KVQ_CORRECTION_EXACT)) return KVQ_ERR_INVALID_ARG;   // one form or the other
   return KVQ_OK;
 }
 
@@ -62,7 +63,8 @@ static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur
   const uint32_t kern = flags & KVQ_KERNEL_MASK;
   *err = KVQ_OK;
   if (kern == KVQ_KERNEL_MMA_SYNC) return false;
-  const bool ok = attn_tcgen05_supports(d, m_tokens, n_cur);
+  // the exact correction (a table look-up per score and group) exists in the warp-level kernel only
+  const bool ok = attn_tcgen05_supports(d, m_tokens, n_cur) && !(flags & KVQ_CORRECTION_EXACT);
   if (kern == KVQ_KERNEL_TCGEN05 && !ok) *err = KVQ_ERR_UNSUPPORTED;
   return ok;
 }
@@ -188,7 +190,7 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
   if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
   if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
   if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
-  if (!attn_tcgen05_supports(desc, m_tokens, n_cur)) return KVQ_ERR_UNSUPPORTED;
+  if (!attn_tcgen05_supports(desc, m_tokens, n_cur) || (flags & KVQ_CORRECTION_EXACT)) return KVQ_ERR_UNSUPPORTED;
   if (m_tokens == 0) return KVQ_OK;
   AttnArgs a;
   a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;

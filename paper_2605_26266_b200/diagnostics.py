@@ -18,12 +18,13 @@ from . import binding as B
 
 
 def attention_stealing(cache: "B.Cache", k_cached, v_cached, q, k_cur, v_cur, softmax_scale,
-                       cache_begin: int = 0, cache_len: int | None = None, kernel_flag: int = B.KVQ_KERNEL_AUTO):
+                       cache_begin: int = 0, cache_len: int | None = None, kernel_flag: int = B.KVQ_KERNEL_AUTO,
+                       exact: bool = True):
     """k_cached, v_cached: the BF16 tensors [batch, heads, n, head_dim] whose quantized form is the window
     [cache_begin, cache_begin + n) of `cache`.  Returns a dict of per-row tensors [batch, heads, rows]:
-    `p_s_ref`, `p_s_uncorrected`, `p_s_corrected`, their differences `dps_uncorrected`, `dps_corrected`
-    (Eq. (9)), and `mse_uncorrected`, `mse_corrected` (mean squared error of the output rows against the
-    unquantized cache)."""
+    `p_s_ref`, `p_s_uncorrected`, `p_s_corrected`, `p_s_exact` (Taylor correction of Eq. (15), exact one of
+    Eq. (12)), their differences to the reference `dps_*` (Eq. (9)), and `mse_*` (mean squared error of the
+    output rows against the unquantized cache)."""
     n = k_cached.shape[2]
     n_cache = n if cache_len is None else cache_len
     assert n_cache == n, "the BF16 copy must cover exactly the attended window"
@@ -41,9 +42,14 @@ def attention_stealing(cache: "B.Cache", k_cached, v_cached, q, k_cur, v_cur, so
     p_s_ref = 1.0 - torch.exp(lse_cur - lse_all)             # P_S = Z_S / (Z_S + Z_R) = 1 - Z_R / Z
 
     res = {"p_s_ref": p_s_ref}
-    for name, flag in (("uncorrected", B.KVQ_CORRECTION_OFF), ("corrected", B.KVQ_CORRECTION_ON)):
+    for name, flag in (("uncorrected", B.KVQ_CORRECTION_OFF), ("corrected", B.KVQ_CORRECTION_ON),
+                       ("exact", B.KVQ_CORRECTION_EXACT)):
+        if flag == B.KVQ_CORRECTION_EXACT and not exact:
+            continue
         mass = torch.empty(shape, **f32)
-        out = B.kvq_attn_corrected(cache, q, k_cur, v_cur, softmax_scale, flag | kernel_flag,
+        # the exact form of Eq. (12) exists in the warp-level kernel only
+        out = B.kvq_attn_corrected(cache, q, k_cur, v_cur, softmax_scale,
+                                   flag | (B.KVQ_KERNEL_AUTO if flag == B.KVQ_CORRECTION_EXACT else kernel_flag),
                                    cache_begin=cache_begin, cache_len=n_cache, cached_mass=mass)
         res["p_s_" + name] = mass
         res["dps_" + name] = mass - p_s_ref

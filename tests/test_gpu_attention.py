@@ -232,3 +232,31 @@ def test_pipeline_config_steps(B):
         B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
         n = O.quantize_append(o, n, sel(k), sel(v))
     T.assert_cache_equal(T.gpu_cache_arrays(g, n), o, n, units=units)
+
+
+@pytest.mark.parametrize("d,bits,group,dist", [(128, 2, 32, "student_t3"), (128, 2, 128, "normal"), (64, 4, 64, "normal")])
+def test_exact_correction_matches_the_oracle(B, d, bits, group, dist):
+    """KVQ_CORRECTION_EXACT: the bias of Eq. (12) (warp-level kernel, a table over the 127 E4M3 step values) against
+    the oracle's exact form, on inputs where it differs visibly from the Taylor form."""
+    w = inputs.Workload("exact", 610 + d + group, 1, 2, d, 140, 0, bits, group, 4, k_dist=dist, k_outliers=8, k_outlier_scale=10.0)
+    g, o, n, sel = _build(B, w, 3, tokens=100, cap=384)
+    q, kc, vc = inputs.make_chunk(w, 6)
+    qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+    sigma = T.sigma_of(d)
+    want = O.attn_corrected(o, 0, n, q, kc, vc, sigma, correction=True, exact=True)
+    taylor = O.attn_corrected(o, 0, n, q, kc, vc, sigma, correction=True)
+    mass = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
+    out = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_EXACT, cached_mass=mass)
+    torch.cuda.synchronize()
+    got = T.from_dev_bf16(out).reshape(want["out"].shape)
+    T.assert_attn_close(got, want["out"], "exact correction")
+    assert np.abs(mass.cpu().numpy().reshape(want["cached_mass"].shape) - want["cached_mass"]).max() < 1e-2
+    if dist == "student_t3":      # here the two forms are far apart, so the test cannot pass by computing the Taylor one
+        assert np.abs(taylor["cached_mass"] - want["cached_mass"]).max() > 0.05
+    # the tcgen05 kernel does not have it
+    with pytest.raises(B.KvqError) as e:
+        B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_EXACT | B.KVQ_KERNEL_TCGEN05)
+    assert e.value.status == B.KVQ_ERR_UNSUPPORTED
+    with pytest.raises(B.KvqError) as e:
+        B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_EXACT | B.KVQ_CORRECTION_ON)
+    assert e.value.status == B.KVQ_ERR_INVALID_ARG
