@@ -5,8 +5,8 @@
 // values (TMA straight into the 128-byte-swizzled operand layout, unrotated query, no bias),
 // then the cached keys and values, which four "dequant" warps expand from the packed
 // 2-/4-bit codes into the same operand layout in shared memory (never to HBM).  Between the
-// two segments the same warps rotate the query tile in place (Hadamard, FP32 butterflies),
-// and compute the per-group squared norms nu of Algorithm 1.
+// two segments the rotated query tile (Hadamard, FP32 butterflies) and the per-group squared norms nu
+// of Algorithm 1, both written by a small pre-pass kernel of the same call, replace the unrotated tile.
 //
 // Score of a cached key (Eq. (15) / Eq. (25)):  s = sigma*q~.k^ - (sigma^2/24) sum_j step_j^2 nu_j.
 // The bias is folded into the score contraction as one extra K=16 MMA step per tile:
@@ -24,13 +24,15 @@
 // Roles (512 threads): warp 0 lane 0 issues TMA; warp 1 runs the MMA schedule converged and one elected
 // lane issues every tcgen05.mma; warps 4-11 are the softmax warps: warp 4+q and warp 8+q share TMEM lanes
 // 32q..32q+31 (one query row per lane) and take columns [0,64) and [64,128) of each score tile, exchanging
-// their partial row maxima through shared memory, for both query tiles in turn; warps 12-15 dequantize
-// and rotate.  Registers are re-split between the roles with setmaxnreg.
+// their partial row maxima through shared memory, for both query tiles in turn; warps 12-15 dequantize.
+// Registers are re-split between the roles with setmaxnreg.  The roles' loops are written to stay small:
+// the SM's instruction cache, and the GPC-level one behind it, bound this kernel before any pipe does.
 //
-// Work is cut into units (batch*head, 256-row query block) of `tiles` key tiles each.  When units are
-// plentiful a CTA computes one whole unit; otherwise the unit x tile steps are divided evenly over one CTA
-// per SM, a CTA walks its range segment by segment, split units leave unnormalised partial results
-// (O, running max, row sums) in the caller's workspace and a small second kernel merges them.
+// Work is cut into units (batch*head, 256-row query block) of `tiles` key tiles each.  Persistent CTAs take
+// whole units in rounds; where that would leave SMs idle (a short last round, or fewer units than SMs) the
+// unit x tile steps are divided evenly over one CTA per SM instead, a CTA walks its range segment by
+// segment, split units leave partial results (their own normalised rows, running max, row sums) in the
+// caller's workspace and a small kernel merges them.
 //
 // Every wait on an mbarrier is bounded: on expiry the CTA records a diagnostic in the caller's status
 // word, all roles leave their loops, in-flight work is drained with a bounded wait, TMEM is freed and the
@@ -73,7 +75,6 @@ constexpr uint32_t kDrainCycles = 20000000u;
 constexpr float kLog2e = 1.4426950408889634f;
 // registers per thread after reallocation: 128 * 72 + 256 * 168 + 128 * 96 = 64512 <= 65536
 constexpr int kRegsIssue = 72, kRegsSoftmax = 168, kRegsDequant = 96;
-constexpr uint32_t kFmaPipePairs = 0x00000000u;      // which of a thread's 32 score pairs use exp2_fma_pipe
 constexpr float kRescaleThreshold = 8.0f;          // lazy rescale of O: only when the max grows by > 2^8
 
 struct TParams {
@@ -173,21 +174,6 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-// 2^x for a pair on the FMA pipe instead of the MUFU: round-to-nearest split x = n + r, |r| <= 1/2, a cubic
-// for 2^r (relative error 7.5e-5, well below BF16 resolution of the probabilities) and an integer add of
-// n into the exponent field.  Inputs are clamped at -126 (results that small are zero for our purposes).
-__device__ __forceinline__ float2 exp2_fma_pipe(float2 x) {
-  x.x = fmaxf(x.x, -126.f); x.y = fmaxf(x.y, -126.f);
-  const float kMagic = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
-  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
-  const float2 r = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-  float2 q = __ffma2_rn(make_float2(0.05517164617776871f, 0.05517164617776871f), r, make_float2(0.2426111251115799f, 0.2426111251115799f));
-  q = __ffma2_rn(q, r, make_float2(0.6932609677314758f, 0.6932609677314758f));
-  q = __ffma2_rn(q, r, make_float2(0.9999280571937561f, 0.9999280571937561f));
-  return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23)),
-                     __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23)));
 }
 __device__ __forceinline__ uint32_t hfma2_f16(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t d;
@@ -773,8 +759,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int i = 0; i < 64; i += 2) {
             const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), c2, nm2);
-            // the MUFU pipe (16 ex2 per clock per SM) is the scarcer unit: a fixed share of the pairs goes to the FMA pipe
-            const float2 pr = ((kFmaPipePairs >> (i >> 1)) & 1u) ? exp2_fma_pipe(x) : make_float2(ex2(x.x), ex2(x.y));
+            const float2 pr = make_float2(ex2(x.x), ex2(x.y));
             sum2 = __fadd2_rn(sum2, pr);
             sr[i >> 1] = cvt_bf16x2(pr.x, pr.y);
           }
@@ -846,7 +831,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
     tc_fence_before();
   } else {
-    // ================= dequant + query rotation =================
+    // ================= dequant warps =================
     setmaxnreg_dec<kRegsDequant>();
     const int dt = tid - 12 * 32;          // 0..127: the key of the tile this thread expands
     Schedule sch(blockIdx.x, gridDim.x, p);
