@@ -261,8 +261,9 @@ def main():
         hq, hk, hv = (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory() for a in (qh, kh, vh))
         hout = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
         dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-        e2e_recs = []
         n_e2e = max(3, min(args.steps, 20))
+        # (a) one step at a time: copy in, attend, append, copy out, all on one stream
+        e2e_recs = []
         barrier()
         for i in range(n_e2e + 3):
             flush.zero_()
@@ -276,7 +277,48 @@ def main():
             if i >= 3:
                 e2e_recs.append((e0, e1))
         barrier()
-        e2e_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in e2e_recs]))
+        e2e_serial_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in e2e_recs]))
+        # (b) the way a caller streams chunks: the next step's host-to-device copies and the previous step's
+        # device-to-host copy run on their own streams beside this step's kernels (two sets of device buffers);
+        # the L2 flush sits on the compute stream inside the timed region
+        s_in, s_out, s_cmp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+        bufs = [(dq, dk, dv, out), (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v), torch.empty_like(out))]
+        houts = [hout, torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()]
+
+        def pipelined(n):
+            ev_in = [torch.cuda.Event() for _ in range(n)]
+            ev_cmp = [torch.cuda.Event() for _ in range(n)]
+            ev_out = [torch.cuda.Event() for _ in range(n)]
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record(s_cmp)
+            s_in.wait_event(t0); s_out.wait_event(t0)
+            for i in range(n):
+                bq, bk, bv, bo = bufs[i & 1]
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(ev_cmp[i - 2])          # the kernels that read this input set are done
+                    bq.copy_(hq, non_blocking=True); bk.copy_(hk, non_blocking=True); bv.copy_(hv, non_blocking=True)
+                    ev_in[i].record(s_in)
+                s_cmp.wait_event(ev_in[i])
+                if i >= 2:
+                    s_cmp.wait_event(ev_out[i - 2])             # this output buffer has been copied out
+                flush.zero_()
+                B.kvq_attn_corrected(cache, bq, bk, bv, sigma, flags, cache_len=n_cached, out=bo, status_word=status)
+                B.kvq_quantize_append(cache, bk, bv, cache_len=n_cached)
+                ev_cmp[i].record(s_cmp)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_cmp[i])
+                    houts[i & 1].copy_(bo, non_blocking=True)
+                    ev_out[i].record(s_out)
+            s_cmp.wait_event(ev_out[n - 1]); s_cmp.wait_event(ev_in[n - 1])
+            t1.record(s_cmp)
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1) / n
+
+        pipelined(4)
+        barrier()
+        e2e_ms = pipelined(n_e2e)
+        barrier()
     # ---- reduce over ranks: slowest rank's time ----
     step_ms, attn_mean, app_mean, attn_off_ms, e2e_ms = replicas.max_over_ranks(
         [step_ms, float(attn_ms.mean()), float(app_ms.mean()), attn_off_ms, 0.0 if args.no_e2e else e2e_ms], device=dev)
@@ -309,6 +351,8 @@ def main():
         }
         if not args.no_e2e:
             res["e2e"] = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                          "mode": "host copies on their own streams beside the kernels (two buffer sets), L2 flush inside",
+                          "serial_ms_per_step": e2e_serial_ms,
                           "h2d_bytes_per_step": int(3 * q.numel() * 2), "d2h_bytes_per_step": int(out.numel() * 2),
                           "ms_per_step": e2e_ms}
         if world == 1 and not args.no_cpu_baseline:
