@@ -209,6 +209,8 @@ class Cache:
     capacity: int
     rotate_k: bool = True
     signs: np.ndarray | None = None
+    rotate_v: bool = False  # values rotated too before quantization (the value path of the rotation scheme the
+                            # paper extends in App. F); the attention output is rotated back
     ring: bool = False      # sliding-window use (Sec. 2: attend to the last n cached chunks): token t lives in slot t mod capacity
 
     def slots(self, begin, n):
@@ -249,6 +251,8 @@ def quantize_append(cache: Cache, cache_len: int, k_bits, v_bits):
     if cache.rotate_k:
         k = rotate_f32_steps(k, cache.signs)
     kc, ks, kz = quantize_vectors(k, cache.bits, cache.group)
+    if cache.rotate_v:
+        v = rotate_f32_steps(v, cache.signs)
     vc, vs, vz = quantize_vectors(v, cache.bits, cache.group)
     cache.k_codes[:, :, sl] = pack_codes(kc, cache.bits)
     cache.v_codes[:, :, sl] = pack_codes(vc, cache.bits)
@@ -303,7 +307,7 @@ def exact_bias(q_rot, key_scale, group, sigma):
 
 def attn_corrected_head(q_bits, kcur_bits, vcur_bits, k_codes, k_scale, k_zero,
                         v_codes, v_scale, v_zero, bits, group, sigma, correction=True,
-                        rotate=True, signs=None, rows=None, exact=False):
+                        rotate=True, signs=None, rows=None, exact=False, rotate_v=False):
     """One (batch, head) unit of Algorithm 1.
 
     q_bits [M, d], kcur_bits/vcur_bits [N_R, d] BF16 bit patterns; cache slices for
@@ -337,7 +341,13 @@ def attn_corrected_head(q_bits, kcur_bits, vcur_bits, k_codes, k_scale, k_zero,
     e = np.exp(s - mx)
     z = e.sum(axis=1, keepdims=True)
     p = e / z
-    out = p[:, :n_s] @ v_hat + p[:, n_s:] @ vr
+    o_s = p[:, :n_s] @ v_hat
+    if rotate_v:
+        # the cached values are stored rotated: R v with R = (1/sqrt d) H diag(s), R^-1 y = s * ((1/sqrt d) H y)
+        o_s = rotate_f64(o_s, None)
+        if signs is not None:
+            o_s = o_s * np.asarray(signs, dtype=np.float64)
+    out = o_s + p[:, n_s:] @ vr
     return {"out": out, "lse": (mx + np.log(z))[:, 0],
             "cached_mass": p[:, :n_s].sum(axis=1), "current_mass": p[:, n_s:].sum(axis=1)}
 
@@ -357,7 +367,7 @@ def attn_corrected(cache: Cache, cache_begin, cache_len, q_bits, kcur_bits, vcur
             cache.k_codes[b, h, sl], cache.k_scale[b, h, sl], cache.k_zero[b, h, sl],
             cache.v_codes[b, h, sl], cache.v_scale[b, h, sl], cache.v_zero[b, h, sl],
             cache.bits, cache.group, sigma, correction, cache.rotate_k, cache.signs,
-            rows, exact)
+            rows, exact, cache.rotate_v)
         outs.append(r["out"])
         lses.append(r["lse"])
         masses.append(r["cached_mass"])

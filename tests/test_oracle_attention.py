@@ -235,6 +235,36 @@ def test_ring_cache_is_the_sliding_window():
             pass
 
 
+def test_rotated_values_equal_the_unrotated_path_on_prerotated_inputs():
+    """rotate_v: quantizing R v and rotating the cached part of the output back must equal what the plain path
+    gives when it is handed values rotated beforehand with a library Hadamard matrix (exact in FP64 here: the
+    entries are small integers / 4, so R v needs no rounding) and its cached output is rotated back by hand."""
+    d, bits, group = 64, 4, 32
+    r = np.random.default_rng(5)
+    signs = r.choice([-1, 1], size=d).astype(np.int8)
+    Hn = scipy.linalg.hadamard(d) / math.sqrt(d)
+    R = Hn * signs[None, :]                                   # R v = H (s * v)
+    ints = lambda shape: r.integers(-8, 9, size=shape).astype(np.float32) * 0.25
+    k, v, q, kc, vc = ints((1, 2, 40, d)), ints((1, 2, 40, d)), ints((1, 2, 9, d)), ints((1, 2, 12, d)), ints((1, 2, 12, d))
+    b = inputs.f32_to_bf16_bits
+    v_rot = np.einsum("ij,bhnj->bhni", R, v.astype(np.float64))
+    assert np.array_equal(O.bf16_bits_to_f64(b(v_rot.astype(np.float32))), v_rot)       # representable: no rounding hidden here
+    a = O.Cache(1, 2, d, bits, group, 128, signs=signs, rotate_v=True)
+    p = O.Cache(1, 2, d, bits, group, 128, signs=signs)
+    O.quantize_append(a, 0, b(k), b(v))
+    O.quantize_append(p, 0, b(k), b(v_rot.astype(np.float32)))
+    for name in ("v_codes", "v_scale", "v_zero", "k_codes"):
+        assert np.array_equal(getattr(a, name), getattr(p, name)), name
+    got = O.attn_corrected(a, 0, 40, b(q), b(kc), b(vc), 0.125)
+    # plain path twice: cached part alone (current values zero) and current part alone, then R^-1 on the cached part
+    zeros = np.zeros_like(vc)
+    cached = O.attn_corrected(p, 0, 40, b(q), b(kc), b(zeros), 0.125)["out"]
+    allv = O.attn_corrected(p, 0, 40, b(q), b(kc), b(vc), 0.125)["out"]
+    want = (cached @ Hn) * signs[None, None, :] + (allv - cached)
+    assert np.abs(got["out"] - want).max() < 1e-12
+    assert np.array_equal(got["cached_mass"], O.attn_corrected(p, 0, 40, b(q), b(kc), b(vc), 0.125)["cached_mass"])
+
+
 def _brute_force(q_bits, kc_bits, vc_bits, cache, n_s, sigma, correction):
     """Algorithm 1 with Python loops, its own dequantization from the stored bytes and
     an explicit Hadamard matrix.  Written separately from the oracle."""
