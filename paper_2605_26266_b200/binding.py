@@ -21,6 +21,7 @@ KVQ_ERR_INVALID_ARG, KVQ_ERR_UNSUPPORTED, KVQ_ERR_ALIGNMENT = -1, -2, -3
 KVQ_ERR_CAPACITY, KVQ_ERR_CUDA, KVQ_ERR_TIMEOUT, KVQ_ERR_WORKSPACE = -4, -5, -6, -7
 KVQ_ROTATE_K = 1
 KVQ_RING = 2
+KVQ_ROTATE_V = 4
 KVQ_CORRECTION_OFF, KVQ_CORRECTION_ON, KVQ_CORRECTION_EXACT = 0, 1, 2
 KVQ_KERNEL_AUTO, KVQ_KERNEL_MMA_SYNC, KVQ_KERNEL_TCGEN05 = 0, 1 << 8, 2 << 8
 
@@ -114,9 +115,10 @@ class Cache:
     """Caller-side owner of the six device buffers of one quantized cache plus its descriptor."""
 
     def __init__(self, batch, heads, head_dim, bits, group, capacity, rotate_k=True, signs=None, device="cuda",
-                 ring=False):
+                 ring=False, rotate_v=False):
         self.desc = kvq_cache_desc(batch, heads, head_dim, bits, group,
-                                   (KVQ_ROTATE_K if rotate_k else 0) | (KVQ_RING if ring else 0), capacity)
+                                   (KVQ_ROTATE_K if rotate_k else 0) | (KVQ_RING if ring else 0)
+                                   | (KVQ_ROTATE_V if rotate_v else 0), capacity)
         sizes = kvq_cache_bytes(self.desc)
         self.buffers = [torch.zeros(n, dtype=torch.uint8, device=device) for n in sizes]
         (self.desc.k_codes, self.desc.v_codes, self.desc.k_scale, self.desc.v_scale,

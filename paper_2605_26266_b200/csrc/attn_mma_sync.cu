@@ -24,7 +24,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 struct AParams {
   const uint16_t* q; const uint16_t* kc; const uint16_t* vc; uint16_t* out;
-  int64_t q_sb, q_sh, q_st, kv_sb, kv_sh, kv_st, o_sb, o_sh, o_st;
+  int64_t q_sb, q_sh, q_st, kv_sb, kv_sh, kv_st, v_sb, v_sh, v_st, o_sb, o_sh, o_st;
   const uint8_t* k_codes; const uint8_t* v_codes; const uint8_t* k_scale; const uint8_t* v_scale;
   const uint16_t* k_zero; const uint16_t* v_zero;
   const int8_t* signs;
@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
       if (kidx < p.n_cur) {
         const int64_t off = (int64_t)b * p.kv_sb + (int64_t)h * p.kv_sh + (int64_t)kidx * p.kv_st + half * (D / 2);
         const uint4* gk = reinterpret_cast<const uint4*>(p.kc + off);
-        const uint4* gv = reinterpret_cast<const uint4*>(p.vc + off);
+        const uint4* gv = reinterpret_cast<const uint4*>(p.vc + (int64_t)b * p.v_sb + (int64_t)h * p.v_sh + (int64_t)kidx * p.v_st + half * (D / 2));
 #pragma unroll
         for (int i = 0; i < D / 16; ++i) { dk[i] = __ldg(gk + i); dv[i] = __ldg(gv + i); }
       } else {
@@ -428,6 +428,7 @@ int launch_attn_mma_sync(const AttnArgs& a) {
   p.vc = static_cast<const uint16_t*>(a.v_cur); p.out = static_cast<uint16_t*>(a.out);
   p.q_sb = a.qs.b; p.q_sh = a.qs.h; p.q_st = a.qs.t;
   p.kv_sb = a.kvs.b; p.kv_sh = a.kvs.h; p.kv_st = a.kvs.t;
+  p.v_sb = a.vs.b; p.v_sh = a.vs.h; p.v_st = a.vs.t;
   p.o_sb = a.os.b; p.o_sh = a.os.h; p.o_st = a.os.t;
   p.k_codes = static_cast<const uint8_t*>(d->k_codes); p.v_codes = static_cast<const uint8_t*>(d->v_codes);
   p.k_scale = static_cast<const uint8_t*>(d->k_scale); p.v_scale = static_cast<const uint8_t*>(d->v_scale);

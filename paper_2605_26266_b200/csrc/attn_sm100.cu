@@ -1122,7 +1122,7 @@ static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t
   CUtensorMap mq, mqr, mk, mv;
   if ((r = make_map(enc, &mq, a.q, a.qs, a.m_tokens, d->heads, d->batch)) != KVQ_OK) return r;
   if ((r = make_map(enc, &mk, a.k_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
-  if ((r = make_map(enc, &mv, a.v_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
+  if ((r = make_map(enc, &mv, a.v_cur, a.vs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
   if ((int64_t)d->batch * d->heads > 65535) return KVQ_ERR_UNSUPPORTED;   // second grid dimension of the pre-pass
   RotParams rp{};
   mqr = mq;                                                  // never read when there are no cached keys

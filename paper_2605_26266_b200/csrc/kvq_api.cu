@@ -19,7 +19,7 @@ int check_shape(const kvq_cache_desc* d) {
   if (d->bits != 2 && d->bits != 4) return KVQ_ERR_UNSUPPORTED;
   if (d->group != 32 && d->group != 64 && d->group != 128) return KVQ_ERR_UNSUPPORTED;
   if (d->capacity % 128 != 0) return KVQ_ERR_INVALID_ARG;
-  if (d->flags & ~(KVQ_ROTATE_K | KVQ_RING)) return KVQ_ERR_INVALID_ARG;
+  if (d->flags & ~(KVQ_ROTATE_K | KVQ_ROTATE_V | KVQ_RING)) return KVQ_ERR_INVALID_ARG;
   return KVQ_OK;
 }
 
@@ -57,6 +57,14 @@ static int check_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t
   if (flags & ~(KVQ_CORRECTION_ON | KVQ_CORRECTION_EXACT | KVQ_KERNEL_MASK)) return KVQ_ERR_INVALID_ARG;
   if ((flags & KVQ_CORRECTION_ON) && (flags & KVQ_CORRECTION_EXACT)) return KVQ_ERR_INVALID_ARG;   // one form or the other
   return KVQ_OK;
+}
+
+// KVQ_ROTATE_V: bytes at the front of the workspace for the rotated copy of the current chunk's values
+// (dense [batch, heads, n_cur, head_dim] BF16, rounded up to 256).  Nothing without cached keys: the output
+// then never leaves the unrotated space.
+static size_t rotv_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur) {
+  if (!(d->flags & KVQ_ROTATE_V) || cache_len <= 0 || m_tokens <= 0) return 0;
+  return ((size_t)d->batch * d->heads * (size_t)n_cur * d->head_dim * 2 + 255) / 256 * 256;
 }
 
 static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur, uint32_t flags, int* err) {
@@ -125,7 +133,7 @@ int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_bytes = tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0;
+  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0);
   return KVQ_OK;
 }
 
@@ -137,7 +145,8 @@ int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_count = tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur) : (m_tokens > 0 ? 1 : 0);
+  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur) : (m_tokens > 0 ? 1 : 0)) +
+               (rotv_bytes(desc, cache_len, m_tokens, n_cur) ? 2 : 0);      // value pre-pass and output post-pass
   return KVQ_OK;
 }
 
@@ -158,8 +167,9 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  if (tc) {
-    const size_t need = attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur);
+  const size_t rotv = rotv_bytes(desc, cache_len, m_tokens, n_cur);
+  {
+    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0);
     if (need > 0) {
       if (!workspace || workspace_bytes < need) return KVQ_ERR_WORKSPACE;
       if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return KVQ_ERR_ALIGNMENT;
@@ -168,12 +178,21 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   if (m_tokens == 0) return KVQ_OK;
   AttnArgs a;
   a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;
-  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides;
+  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides; a.vs = kv_strides;
   a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out_bf16; a.os = o_strides;
   a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse_out; a.cached_mass = cached_mass_out;
   a.workspace = workspace; a.workspace_bytes = workspace_bytes; a.status_word = status_word;
   a.stream = (cudaStream_t)stream;
-  return tc ? launch_attn_tcgen05(a) : launch_attn_mma_sync(a);
+  if (rotv) {
+    // values are cached rotated: bring the current chunk's values into the same space, attend, rotate the output back
+    const kvq_strides dense{(int64_t)desc->heads * n_cur * desc->head_dim, n_cur * (int64_t)desc->head_dim, (int64_t)desc->head_dim};
+    if ((r = launch_rotate_rows(desc, v_cur, kv_strides, workspace, dense, n_cur, false, a.stream)) != KVQ_OK) return r;
+    a.v_cur = workspace; a.vs = dense;
+    a.workspace = static_cast<uint8_t*>(workspace) + rotv; a.workspace_bytes = workspace_bytes - rotv;
+  }
+  r = tc ? launch_attn_tcgen05(a) : launch_attn_mma_sync(a);
+  if (r == KVQ_OK && rotv) r = launch_rotate_rows(desc, out_bf16, o_strides, out_bf16, o_strides, m_tokens, true, a.stream);
+  return r;
 }
 
 int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
@@ -190,11 +209,12 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
   if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
   if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
   if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
-  if (!attn_tcgen05_supports(desc, m_tokens, n_cur) || (flags & KVQ_CORRECTION_EXACT)) return KVQ_ERR_UNSUPPORTED;
+  if (!attn_tcgen05_supports(desc, m_tokens, n_cur) || (flags & KVQ_CORRECTION_EXACT) || (desc->flags & KVQ_ROTATE_V))
+    return KVQ_ERR_UNSUPPORTED;
   if (m_tokens == 0) return KVQ_OK;
   AttnArgs a;
   a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;
-  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides;
+  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides; a.vs = kv_strides;
   a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out_bf16; a.os = o_strides;
   a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse_out; a.cached_mass = cached_mass_out;
   a.workspace = nullptr; a.workspace_bytes = 0; a.status_word = status_word;

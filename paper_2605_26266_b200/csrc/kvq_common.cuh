@@ -36,7 +36,8 @@ struct AttnArgs {
   const kvq_cache_desc* desc;
   int64_t cache_begin, cache_len;
   const void* q; kvq_strides qs;
-  const void* k_cur; const void* v_cur; kvq_strides kvs;
+  const void* k_cur; const void* v_cur; kvq_strides kvs;   // strides of k_cur
+  kvq_strides vs;                                            // strides of v_cur
   int64_t m_tokens, n_cur;
   void* out; kvq_strides os;
   float softmax_scale;
@@ -47,6 +48,9 @@ struct AttnArgs {
   cudaStream_t stream;
 };
 int launch_attn_mma_sync(const AttnArgs& a);
+// y = (1/sqrt d) H (signs . x) per row (inverse: x = signs . ((1/sqrt d) H y)), BF16 [batch, heads, tokens, head_dim]
+int launch_rotate_rows(const kvq_cache_desc* d, const void* src, kvq_strides ss, void* dst, kvq_strides ds,
+                       int64_t tokens, bool inverse, cudaStream_t st);
 // tcgen05 kernel: returns KVQ_ERR_UNSUPPORTED for shapes it does not cover.
 bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur);
 size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);

@@ -24,7 +24,7 @@ struct QParams {
   const uint16_t* k; const uint16_t* v;
   int64_t sb, sh, st;          // element strides of k and v
   int64_t n_tokens, cache_len, capacity;
-  int heads, group, rotate;
+  int heads, group, rotate, rotate_v;
   const int8_t* signs;
   uint8_t* codes[2]; uint8_t* scale[2]; uint16_t* zero[2];
   int tiles_per_bh;
@@ -239,6 +239,13 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
     }
     quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[0], s_scale[0], s_zero[0]);
     decode_vec<EPL>(rv_cur, x);
+    if (p.rotate_v) {                                       // values stored rotated too (KVQ_ROTATE_V)
+      if (p.signs) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], (float)p.signs[l8 * EPL + e]);
+      }
+      hadamard<EPL>(x, l8, c_d);
+    }
     quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[1], s_scale[1], s_zero[1]);
     __syncthreads();
     // The tile goes to slots slot0 .. slot0 + nt - 1, modulo the capacity: one piece, or two when a ring
@@ -289,6 +296,7 @@ int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const voi
   p.sb = kv.b; p.sh = kv.h; p.st = kv.t;
   p.n_tokens = n_tokens; p.cache_len = cache_len % d->capacity; p.capacity = d->capacity;
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
+  p.rotate_v = (d->flags & KVQ_ROTATE_V) ? 1 : 0;
   p.signs = d->signs;
   p.codes[0] = static_cast<uint8_t*>(d->k_codes); p.codes[1] = static_cast<uint8_t*>(d->v_codes);
   p.scale[0] = static_cast<uint8_t*>(d->k_scale); p.scale[1] = static_cast<uint8_t*>(d->v_scale);
