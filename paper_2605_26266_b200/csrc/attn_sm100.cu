@@ -914,8 +914,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 }
 
 // Combines the partial results of every unit whose key tiles were split over several CTAs.
-// grid (n_units - n_whole, 32): a block handles 8 rows x 128 columns; thread = (row, 8-column group).
-__global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_ctas) {
+// grid (n_units - n_whole, 4): a block handles 64 rows x 128 columns, 16 rows at a time; thread = (row, 8-column group).
+__global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_ctas) {
   const int unit = p.n_whole + blockIdx.x;
   const int T = p.tiles;
   // Which CTAs worked on this unit, found once per block (64-bit divisions): CTA c owns the tile steps
@@ -941,32 +941,50 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_
   __syncthreads();
   const int c_first = s_first, c_last = s_last, first_slot = s_first_slot;
   if (c_first == c_last) return;                       // the unit was computed whole by one CTA
-  const int r256 = blockIdx.y * 8 + (threadIdx.x >> 4);
   const int cg = threadIdx.x & 15;
   const int bh = unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+  const int r256 = blockIdx.y * 64 + pass * 16 + (threadIdx.x >> 4);
   const int row = (unit - bh * p.q_blocks) * 256 + r256;
-  if (row >= p.m_tokens) return;
+  if (row >= p.m_tokens) break;
+  // Partials are taken four at a time with all of their loads issued before any is used: a thread moves only
+  // 16 bytes per partial, so the kernel lives on loads in flight.
+  auto slot_of = [&](int c) { return p.partial + (size_t)(2 * c + (c == c_first ? first_slot : 0)) * kSlotBytes; };
   float m = -INFINITY;
-  for (int c = c_first; c <= c_last; ++c) {
-    const int slot = 2 * c + (c == c_first ? first_slot : 0);
-    m = fmaxf(m, reinterpret_cast<const float*>(p.partial + (size_t)slot * kSlotBytes + kSlotStats)[r256]);
+  for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+    float mm[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      mm[j] = (c0 + j <= c_last) ? reinterpret_cast<const float*>(slot_of(c0 + j) + kSlotStats)[r256] : -INFINITY;
+    m = fmaxf(fmaxf(m, fmaxf(mm[0], mm[1])), fmaxf(mm[2], mm[3]));
   }
   // out = sum_i w_i O_i / sum_i w_i with w_i = l_i 2^(m_i - m): every partial row is already normalised by its l_i
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   float l_cur = 0.f, l_cac = 0.f;
-  for (int c = c_first; c <= c_last; ++c) {
-    const int slot = 2 * c + (c == c_first ? first_slot : 0);
-    const uint8_t* sl = p.partial + (size_t)slot * kSlotBytes;
-    const float* st = reinterpret_cast<const float*>(sl + kSlotStats);
-    const float f = exp2f(st[r256] - m);
-    const float lc = f * st[256 + r256], la = f * st[512 + r256];
-    l_cur += lc; l_cac += la;
-    const float w = lc + la;
-    const uint4 a = *reinterpret_cast<const uint4*>(sl + ((size_t)r256 * kD + cg * 8) * 2);
-    acc[0] += w * bf16_bits_to_f32(a.x & 0xFFFFu); acc[1] += w * bf16_bits_to_f32(a.x >> 16);
-    acc[2] += w * bf16_bits_to_f32(a.y & 0xFFFFu); acc[3] += w * bf16_bits_to_f32(a.y >> 16);
-    acc[4] += w * bf16_bits_to_f32(a.z & 0xFFFFu); acc[5] += w * bf16_bits_to_f32(a.z >> 16);
-    acc[6] += w * bf16_bits_to_f32(a.w & 0xFFFFu); acc[7] += w * bf16_bits_to_f32(a.w >> 16);
+  for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+    float sm[4], sc[4], sa[4];
+    uint4 a[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const bool have = c0 + j <= c_last;
+      const uint8_t* sl = slot_of(have ? c0 + j : c_last);
+      const float* st = reinterpret_cast<const float*>(sl + kSlotStats);
+      sm[j] = have ? st[r256] : -INFINITY;                  // weight 2^(-inf) = 0 for the slots that are not there
+      sc[j] = st[256 + r256]; sa[j] = st[512 + r256];
+      a[j] = *reinterpret_cast<const uint4*>(sl + ((size_t)r256 * kD + cg * 8) * 2);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float f = exp2f(sm[j] - m);
+      const float lc = f * sc[j], la = f * sa[j];
+      l_cur += lc; l_cac += la;
+      const float w = lc + la;
+      acc[0] += w * bf16_bits_to_f32(a[j].x & 0xFFFFu); acc[1] += w * bf16_bits_to_f32(a[j].x >> 16);
+      acc[2] += w * bf16_bits_to_f32(a[j].y & 0xFFFFu); acc[3] += w * bf16_bits_to_f32(a[j].y >> 16);
+      acc[4] += w * bf16_bits_to_f32(a[j].z & 0xFFFFu); acc[5] += w * bf16_bits_to_f32(a[j].z >> 16);
+      acc[6] += w * bf16_bits_to_f32(a[j].w & 0xFFFFu); acc[7] += w * bf16_bits_to_f32(a[j].w >> 16);
+    }
   }
   const float l = l_cur + l_cac, inv = 1.0f / l;
   uint4 v;
@@ -977,6 +995,7 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(const TParams p, int n_
     const int64_t idx = (int64_t)bh * p.m_tokens + row;
     if (p.lse) p.lse[idx] = (m + log2f(l)) * 0.6931471805599453f;
     if (p.cached_mass) p.cached_mass[idx] = l_cac * inv;
+  }
   }
 }
 
@@ -1068,7 +1087,7 @@ int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk,
   attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mqr, mk, mv, p);
   KVQ_CUDA_TRY(cudaGetLastError());
   if (p.n_whole != p.n_units) {   // units were split over CTAs: combine their partial results
-    attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 32), 128, 0, st>>>(p, (int)grid.x);
+    attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 4), 256, 0, st>>>(p, (int)grid.x);
     KVQ_CUDA_TRY(cudaGetLastError());
   }
   return KVQ_OK;
