@@ -60,7 +60,8 @@ constexpr int kOffV = kOffK + 2 * kTileBytes;      // 2 stages
 constexpr int kOffAx = kOffV + 2 * kTileBytes;     // 2 query tiles
 constexpr int kOffBx = kOffAx + 2 * kXBytes;       // 2 stages
 constexpr int kOffBar = kOffBx + 2 * kXBytes;
-constexpr int kNumBars = 30;
+constexpr int kNumBars = 30;                       // mbarriers, 8 bytes each (enum Bar below)
+static_assert(kNumBars * 8 <= 256, "barrier area");
 constexpr int kOffXmax = kOffBar + 256;            // float [2 column halves][256 rows]: row-max exchange
 constexpr int kOffXl = kOffXmax + 2 * 256 * 4;     // float [2][256][2]: row-sum exchange (current, cached)
 constexpr int kOffMisc = kOffXl + 2 * 256 * 2 * 4;
