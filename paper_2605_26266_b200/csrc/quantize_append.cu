@@ -18,7 +18,7 @@ namespace {
 constexpr int kTileTokens = 32;
 constexpr int kWarps = 8;
 constexpr int kTokPerWarp = kTileTokens / kWarps;
-constexpr int kCtasPerSm = 3;      // persistent grid: SMs x this (a multiple of the SM count)
+constexpr int kCtasPerSm = 4;      // persistent grid: SMs x this (a multiple of the SM count)
 
 struct QParams {
   const uint16_t* k; const uint16_t* v;
