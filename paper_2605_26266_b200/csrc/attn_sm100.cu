@@ -60,7 +60,7 @@ constexpr int kOffV = kOffK + 2 * kTileBytes;      // 2 stages
 constexpr int kOffAx = kOffV + 2 * kTileBytes;     // 2 query tiles
 constexpr int kOffBx = kOffAx + 2 * kXBytes;       // 2 stages
 constexpr int kOffBar = kOffBx + 2 * kXBytes;
-constexpr int kNumBars = 30;                       // mbarriers, 8 bytes each (enum Bar below)
+constexpr int kNumBars = 21;                       // mbarriers, 8 bytes each (enum Bar below)
 static_assert(kNumBars * 8 <= 256, "barrier area");
 constexpr int kOffXmax = kOffBar + 256;            // float [2 column halves][256 rows]: row-max exchange
 constexpr int kOffXl = kOffXmax + 2 * 256 * 4;     // float [2][256][2]: row-sum exchange (current, cached)
@@ -68,8 +68,7 @@ constexpr int kOffMisc = kOffXl + 2 * 256 * 2 * 4;
 constexpr int kSmemBytes = kOffMisc + 64 + 1024;   // + slack to align the base to 1024
 
 enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull = 9, kPFull = 11,
-           kODone = 13, kQCurDone = 15, kQRotFull = 16, kDrain = 17, kQEmpty = 18, kOFree = 19,
-           kPair = 21 /* 8: [query tile][lane quarter], the two warps that share 32 rows */ };
+           kODone = 13, kQCurDone = 15, kQRotFull = 16, kDrain = 17, kQEmpty = 18, kOFree = 19 };
 
 constexpr uint32_t kTimeoutCycles = 2000000000u;   // about a second; 32-bit clock differences stay exact below 2^32
 constexpr uint32_t kDrainCycles = 20000000u;
@@ -162,6 +161,13 @@ struct Ctx {
     while (!mbar_try_wait(b, parity) && (uint32_t)clock() - t0 < kDrainCycles) {}
   }
 };
+
+// The two softmax warps that share 32 query rows (warp 4 + q and warp 8 + q) meet at hardware barrier 1 + q to
+// exchange row maxima and row sums: about a third of the latency of an mbarrier round trip, once per query tile
+// and key tile.  Both warps run the same sequence of bounded waits before every meeting, so in a healthy run
+// neither can miss one; pair_release covers the aborting CTA (see the end of the softmax role).
+__device__ __forceinline__ void pair_sync(int q) { asm volatile("bar.sync %0, 64;" :: "r"(1 + q) : "memory"); }
+__device__ __forceinline__ void pair_release(int q) { asm volatile("bar.arrive %0, 64;" :: "r"(1 + q) : "memory"); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
@@ -484,7 +490,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(cx.bar(kQEmpty), 1);
     mbar_init(cx.bar(kOFree + 0), 256);
     mbar_init(cx.bar(kOFree + 1), 256);
-    for (int i = 0; i < 8; ++i) mbar_init(cx.bar(kPair + i), 64);
     fence_barrier_init();
     prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_qr); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
   }
@@ -694,7 +699,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     Schedule sch(blockIdx.x, gridDim.x, p);
     Segment sg;
     int it = 0, nseg = 0;
-    uint32_t pair_phase = 0;                                  // pair barriers flip once per tile and once per epilogue
     bool ok = true;
     while (ok && sch.next(sg)) {
       // Running max and row sums (current / cached keys) of the query tile being worked on (m_a ...) and of
@@ -731,9 +735,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const float mine = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
           xmax[half * 256 + r256] = mine;
           tc_fence_before();
-          mbar_arrive(cx.bar(kPair + qt * 4 + wq));
-          ok = __all_sync(0xFFFFFFFFu, cx.wait(kPair + qt * 4 + wq, pair_phase, 304));
-          if (!ok) break;
+          pair_sync(wq);
           tc_fence_after();
           const float m_new = fmaxf(m_a, fmaxf(mine, xmax[(half ^ 1) * 256 + r256]) * c_row);
           if (__any_sync(0xFFFFFFFFu, m_new - m_a > kRescaleThreshold)) {
@@ -771,7 +773,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mbar_arrive(cx.bar(kPFull + qt));
           { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
         }
-        pair_phase ^= 1;
       }
       if (!ok) break;
       // ---- segment epilogue: read O out of TMEM, release it, combine the two column halves' row sums ----
@@ -792,9 +793,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_arrive(cx.bar(kOFree + qt));
         xl[(half * 256 + r256) * 2] = lcur_a;
         xl[(half * 256 + r256) * 2 + 1] = lcac_a;
-        mbar_arrive(cx.bar(kPair + qt * 4 + wq));
-        ok = __all_sync(0xFFFFFFFFu, cx.wait(kPair + qt * 4 + wq, pair_phase, 305));
-        if (!ok) break;
+        pair_sync(wq);
         const float lc = lcur_a + xl[((half ^ 1) * 256 + r256) * 2];
         const float la = lcac_a + xl[((half ^ 1) * 256 + r256) * 2 + 1];
         const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
@@ -827,9 +826,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
       }
-      pair_phase ^= 1;
       ++nseg;
     }
+    // Leaving because the CTA is aborting: the partner warp may be sitting in pair_sync, which has no time-out
+    // of its own.  One arrival on the pair's barrier lets it through; it then fails its next bounded wait.
+    if (*cx.abort) pair_release(wq);
     tc_fence_before();
   } else {
     // ================= dequant warps =================
