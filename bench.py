@@ -167,7 +167,7 @@ def main():
         sec = float(np.mean(times))
         val = flops / sec / 1e12
         print(json.dumps({
-            "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": 0, "steps": steps,
+            "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus, "gpus_used": 0, "steps": steps,
             "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": sample},
