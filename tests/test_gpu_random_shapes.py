@@ -65,3 +65,35 @@ def test_random_shape(c):
         T.assert_attn_close(T.from_dev_bf16(out).reshape(want["out"].shape), want["out"], kname)
         assert np.abs(lse.cpu().numpy().reshape(want["lse"].shape) - want["lse"]).max() < 2e-2, kname
         assert np.abs(mass.cpu().numpy().reshape(want["cached_mass"].shape) - want["cached_mass"]).max() < 1e-2, kname
+
+
+def _append_cases():
+    r = np.random.default_rng(7)
+    out = []
+    for i in range(16):
+        d = int(r.choice([64, 128]))
+        out.append(dict(i=i, d=d, bits=int(r.choice([2, 4])), group=int(r.choice([g for g in (32, 64, 128) if g <= d])),
+                        batch=int(r.integers(1, 3)), heads=int(r.integers(1, 5)), n=int(r.choice(LENGTHS[:15])),
+                        pos=int(r.integers(0, 200)), rotate=bool(r.integers(0, 2)), rotate_v=bool(r.integers(0, 2)),
+                        ring=bool(r.integers(0, 2)), scale=float(r.choice([1e-3, 1.0, 37.0, 1e4]))))
+    return out
+
+
+@pytest.mark.parametrize("c", _append_cases(), ids=lambda c: f"{c['i']}-d{c['d']}b{c['bits']}g{c['group']}-n{c['n']}p{c['pos']}")
+def test_random_append_bit_exact(c):
+    """Appends of random length at random positions (unaligned destinations, ring wrap) with random magnitudes."""
+    from paper_2605_26266_b200 import binding as B
+    d, cap = c["d"], 384
+    r = np.random.default_rng(100 + c["i"])
+    x = (r.standard_normal((2, c["batch"], c["heads"], c["n"], d)) * c["scale"]).astype(np.float32)
+    x[0, ..., : d // 4] += 3.0 * c["scale"]                      # a shifted block: non-trivial zero-points
+    kb, vb = inputs.f32_to_bf16_bits(x[0]), inputs.f32_to_bf16_bits(x[1])
+    kw = dict(rotate_k=c["rotate"], ring=c["ring"], rotate_v=c["rotate_v"])
+    g = B.Cache(c["batch"], c["heads"], d, c["bits"], c["group"], cap, **kw)
+    o = O.Cache(c["batch"], c["heads"], d, c["bits"], c["group"], cap, **kw)
+    pos = c["pos"] + (cap - 100 if c["ring"] else 0)              # a ring append straddles the end of the buffer
+    if not c["ring"] and pos + c["n"] > cap:
+        pos = cap - c["n"]
+    B.kvq_quantize_append(g, T.to_dev(kb), T.to_dev(vb), cache_len=pos)
+    O.quantize_append(o, pos, kb, vb)
+    T.assert_cache_equal(T.gpu_cache_arrays(g, cap), o, cap)
