@@ -211,6 +211,8 @@ class Cache:
     signs: np.ndarray | None = None
     rotate_v: bool = False  # values rotated too before quantization (the value path of the rotation scheme the
                             # paper extends in App. F); the attention output is rotated back
+    k_per_channel: bool = False  # App. E: key steps and zero-points per channel, shared by the `group` tokens of a
+                            # block (k_scale, k_zero are then [B, H, capacity // group, d]); values stay per token
     ring: bool = False      # sliding-window use (Sec. 2: attend to the last n cached chunks): token t lives in slot t mod capacity
 
     def slots(self, begin, n):
@@ -230,9 +232,9 @@ class Cache:
         nb = d * self.bits // 8
         self.k_codes = np.zeros((B, H, C, nb), np.uint8)
         self.v_codes = np.zeros((B, H, C, nb), np.uint8)
-        self.k_scale = np.zeros((B, H, C, G), np.uint8)
+        self.k_scale = np.zeros((B, H, C // self.group, d) if self.k_per_channel else (B, H, C, G), np.uint8)
         self.v_scale = np.zeros((B, H, C, G), np.uint8)
-        self.k_zero = np.zeros((B, H, C, G), np.uint16)
+        self.k_zero = np.zeros((B, H, C // self.group, d) if self.k_per_channel else (B, H, C, G), np.uint16)
         self.v_zero = np.zeros((B, H, C, G), np.uint16)
 
     @property
@@ -250,15 +252,29 @@ def quantize_append(cache: Cache, cache_len: int, k_bits, v_bits):
     v = bf16_bits_to_f64(v_bits)
     if cache.rotate_k:
         k = rotate_f32_steps(k, cache.signs)
-    kc, ks, kz = quantize_vectors(k, cache.bits, cache.group)
+    if cache.k_per_channel:
+        # App. E: for every block of `group` consecutive tokens and every channel, one step and one zero-point over
+        # the block's tokens: Eq. (1) with the roles of tokens and channels exchanged inside a block
+        g = cache.group
+        if cache_len % g or n % g:
+            raise ValueError("per-channel keys are appended in whole blocks of `group` tokens")
+        kb = np.swapaxes(k.reshape(k.shape[:2] + (n // g, g, k.shape[-1])), -1, -2)      # [B, H, blocks, d, g]
+        kc, ks, kz = quantize_vectors(kb, cache.bits, g)
+        kc = np.swapaxes(kc, -1, -2).reshape(k.shape)
+        blocks = sl[::g] // g
+        cache.k_codes[:, :, sl] = pack_codes(kc, cache.bits)
+        cache.k_scale[:, :, blocks] = ks[..., 0]
+        cache.k_zero[:, :, blocks] = kz[..., 0]
+    else:
+        kc, ks, kz = quantize_vectors(k, cache.bits, cache.group)
+        cache.k_codes[:, :, sl] = pack_codes(kc, cache.bits)
+        cache.k_scale[:, :, sl] = ks
+        cache.k_zero[:, :, sl] = kz
     if cache.rotate_v:
         v = rotate_f32_steps(v, cache.signs)
     vc, vs, vz = quantize_vectors(v, cache.bits, cache.group)
-    cache.k_codes[:, :, sl] = pack_codes(kc, cache.bits)
     cache.v_codes[:, :, sl] = pack_codes(vc, cache.bits)
-    cache.k_scale[:, :, sl] = ks
     cache.v_scale[:, :, sl] = vs
-    cache.k_zero[:, :, sl] = kz
     cache.v_zero[:, :, sl] = vz
     return cache_len + n
 
@@ -307,31 +323,33 @@ def exact_bias(q_rot, key_scale, group, sigma):
 
 def attn_corrected_head(q_bits, kcur_bits, vcur_bits, k_codes, k_scale, k_zero,
                         v_codes, v_scale, v_zero, bits, group, sigma, correction=True,
-                        rotate=True, signs=None, rows=None, exact=False, rotate_v=False):
+                        rotate=True, signs=None, rows=None, exact=False, rotate_v=False, k_group=None):
     """One (batch, head) unit of Algorithm 1.
 
     q_bits [M, d], kcur_bits/vcur_bits [N_R, d] BF16 bit patterns; cache slices for
     the attended window, [N_S, ...].  rows: optional index array of query rows.
     Returns dict(out [m, d], lse [m], cached_mass [m], current_mass [m]); the two masses are
-    P_S and P_R of Eq. (4), summed separately."""
+    P_S and P_R of Eq. (4), summed separately.  k_group: channels per key group if it differs from the values'
+    (1 for per-channel keys, whose k_scale / k_zero arrive expanded to one row per token, [N_S, d])."""
+    k_group = group if k_group is None else k_group
     q = bf16_bits_to_f64(q_bits)
     if rows is not None:
         q = q[rows]
     d = q.shape[-1]
-    G = d // group
+    G = d // k_group
     kr = bf16_bits_to_f64(kcur_bits)
     vr = bf16_bits_to_f64(vcur_bits)
     n_s = k_codes.shape[0]
     q_rot = rotate_f64(q, signs) if rotate else q
-    nu = (q_rot.reshape(q.shape[0], G, group) ** 2).sum(axis=-1)          # Alg. 1: nu[m, j]
+    nu = (q_rot.reshape(q.shape[0], G, k_group) ** 2).sum(axis=-1)        # Alg. 1: nu[m, j]
     s_r = sigma * (q @ kr.T)                                                # S_R
     if n_s > 0:
-        k_hat = dequant(k_codes, k_scale, k_zero, bits, group)              # dequant(K^q)
+        k_hat = dequant(k_codes, k_scale, k_zero, bits, k_group)            # dequant(K^q)
         v_hat = dequant(v_codes, v_scale, v_zero, bits, group)
         s_s = sigma * (q_rot @ k_hat.T)                                     # S_S
         if correction:
             ds = e4m3_decode(k_scale)
-            b = exact_bias(q_rot, ds, group, sigma) if exact else taylor_bias(nu, ds, sigma)
+            b = exact_bias(q_rot, ds, k_group, sigma) if exact else taylor_bias(nu, ds, sigma)
             s_s = s_s - b                                                   # cached scores only
     else:
         s_s = np.zeros((q.shape[0], 0))
@@ -361,13 +379,17 @@ def attn_corrected(cache: Cache, cache_begin, cache_len, q_bits, kcur_bits, vcur
     units = heads if heads is not None else [(b, h) for b in range(B) for h in range(H)]
     sl = cache.slots(cache_begin, cache_len)
     outs, lses, masses, cmasses = [], [], [], []
+    # per-channel keys (App. E): every token takes the steps and zero-points of its block, one per channel; the bias
+    # of Eq. (15) with groups of one channel is then the App. E form (1/24d) sum_c q_c^2 step_c^2, equal for all
+    # tokens of a block
+    ksl = sl // cache.group if cache.k_per_channel else sl
     for (b, h) in units:
         r = attn_corrected_head(
             q_bits[b, h], kcur_bits[b, h], vcur_bits[b, h],
-            cache.k_codes[b, h, sl], cache.k_scale[b, h, sl], cache.k_zero[b, h, sl],
+            cache.k_codes[b, h, sl], cache.k_scale[b, h, ksl], cache.k_zero[b, h, ksl],
             cache.v_codes[b, h, sl], cache.v_scale[b, h, sl], cache.v_zero[b, h, sl],
             cache.bits, cache.group, sigma, correction, cache.rotate_k, cache.signs,
-            rows, exact, cache.rotate_v)
+            rows, exact, cache.rotate_v, 1 if cache.k_per_channel else None)
         outs.append(r["out"])
         lses.append(r["lse"])
         masses.append(r["cached_mass"])

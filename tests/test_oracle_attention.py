@@ -333,3 +333,33 @@ def test_workload_recipes_are_deterministic_and_shaped():
     assert ((kf > 4 * np.median(kf, axis=1, keepdims=True)).sum(axis=1) == 8).all()   # 8 outlier channels
     rows = inputs.sample_rows(1560, 128, 16)
     assert rows[0] == 0 and rows[-1] == 1559 and len(set(rows // 128)) == 13
+
+
+def test_per_channel_keys_bias_is_one_scalar_per_block_and_matches_app_e():
+    """App. E: with per-channel keys the Taylor bias is (sigma^2 / 24) sum_c q_c^2 step_c^2, the same for every
+    token of a block.  Brute force over the stored bytes, with an explicit softmax."""
+    d, bits, g, sigma = 64, 2, 32, 0.125
+    w = inputs.Workload("pc", 88, 1, 1, d, 64, 0, bits, g, 2, k_outliers=2, k_outlier_scale=5.0)
+    c = O.Cache(1, 1, d, bits, g, 128, k_per_channel=True)
+    _, k, v = inputs.make_chunk(w, 0)
+    O.quantize_append(c, 0, k, v)
+    q, kc, vc = inputs.make_chunk(w, 3, tokens=10)
+    got = O.attn_corrected(c, 0, 64, q, kc, vc, sigma)
+    H = scipy.linalg.hadamard(d) / math.sqrt(d)
+    f = O.bf16_bits_to_f64
+    q_rot = f(q)[0, 0] @ H.T
+    codes = O.unpack_codes(c.k_codes[0, 0, :64], bits).astype(np.float64)
+    s = np.zeros((10, 64 + 10))
+    for i in range(64):
+        ds = O.e4m3_decode(c.k_scale[0, 0, i // g])              # [d] steps of the token's block
+        zs = f(c.k_zero[0, 0, i // g])
+        k_hat = (codes[i] - zs) * ds
+        for m in range(10):
+            b = sigma ** 2 / 24.0 * float(np.sum(q_rot[m] ** 2 * ds ** 2))
+            s[m, i] = sigma * float(q_rot[m] @ k_hat) - b
+    s[:, 64:] = sigma * f(q)[0, 0] @ f(kc)[0, 0].T
+    p = np.exp(s - s.max(1, keepdims=True)); p /= p.sum(1, keepdims=True)
+    v_hat = O.dequant(c.v_codes[0, 0, :64], c.v_scale[0, 0, :64], c.v_zero[0, 0, :64], bits, g)
+    want = p[:, :64] @ v_hat + p[:, 64:] @ f(vc)[0, 0]
+    assert np.abs(got["out"][0] - want).max() < 1e-12
+    assert np.abs(got["cached_mass"][0] - p[:, :64].sum(1)).max() < 1e-12

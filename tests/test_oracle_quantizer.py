@@ -174,3 +174,38 @@ def test_fp32_steps_vs_unrounded_informational():
     a, _, _ = O.quantize_vectors(y, 2, 64, fp32_steps=True)
     b, _, _ = O.quantize_vectors(y, 2, 64, fp32_steps=False)
     assert np.mean(a != b) < 1e-4 and np.abs(a - b).max() <= 1
+
+
+def test_per_channel_keys_against_the_scalar_implementation():
+    """App. E layout: one step / zero-point per (block of `group` tokens, channel).  The stored bytes must equal the
+    scalar second implementation run over the `group` tokens of each channel of each block, and the dequantized
+    keys must be (code - zero_c) * step_c."""
+    from paper_2605_26266_b200 import inputs
+    r = np.random.default_rng(3)
+    for bits, g, d in ((2, 32, 64), (4, 64, 128)):
+        n = 2 * g
+        x = (r.standard_normal((1, 2, n, d)) * np.exp(r.uniform(-1, 2, (1, 2, 1, d)))).astype(np.float32)
+        kb = inputs.f32_to_bf16_bits(x)
+        vb = inputs.f32_to_bf16_bits(x[..., ::-1].copy())
+        c = O.Cache(1, 2, d, bits, g, 4 * g, rotate_k=False, k_per_channel=True)
+        assert c.k_scale.shape == (1, 2, 4, d) and c.v_scale.shape == (1, 2, 4 * g, d // g)
+        O.quantize_append(c, g, kb, vb)                         # blocks 1 and 2
+        k = O.bf16_bits_to_f64(kb)
+        codes = O.unpack_codes(c.k_codes[:, :, g:3 * g], bits)
+        for h in range(2):
+            for blk in range(2):
+                for ch in range(0, d, 7):
+                    col = k[0, h, blk * g:(blk + 1) * g, ch]
+                    c2, s2, z2 = _scalar_quantize_f32(col, bits, g)
+                    assert codes[0, h, blk * g:(blk + 1) * g, ch].tolist() == c2
+                    assert int(c.k_scale[0, h, 1 + blk, ch]) == s2[0] and int(c.k_zero[0, h, 1 + blk, ch]) == z2[0]
+        # values keep the per-token layout of the plain cache
+        p = O.Cache(1, 2, d, bits, g, 4 * g, rotate_k=False)
+        O.quantize_append(p, g, kb, vb)
+        assert np.array_equal(p.v_codes, c.v_codes) and np.array_equal(p.v_scale, c.v_scale)
+        # whole blocks only
+        try:
+            O.quantize_append(c, 0, kb[:, :, :g - 1], vb[:, :, :g - 1])
+            raise AssertionError("accepted a partial block")
+        except ValueError:
+            pass
