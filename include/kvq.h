@@ -60,6 +60,11 @@ extern "C" {
                                       path of the rotation scheme App. F extends); kvq_attn_corrected then rotates the
                                       current chunk's values the same way (a pre-pass into the workspace) and rotates
                                       the output back (a post-pass over out).  Not with the static-scratch entry. */
+#define KVQ_K_PER_CHANNEL     8u   /* App. E: key steps and zero-points per channel, shared by the `group` tokens of a
+                                      block: k_scale and k_zero are then [batch,heads,capacity/group,head_dim] (the same
+                                      bytes in all), values keep the per-token layout.  Appends and windows must start
+                                      on multiples of `group` tokens and appends bring whole blocks
+                                      (KVQ_ERR_ALIGNMENT).  Attention: warp-level kernel only, Taylor form only. */
 #define KVQ_RING              2u   /* ring cache for sliding-window attention (Section 2; the windows of Section 5.1):
                                       token t lives in slot t mod capacity, new tokens overwrite the oldest.  Token
                                       positions (cache_len of kvq_quantize_append, cache_begin of the attention calls)
@@ -87,7 +92,7 @@ typedef struct kvq_cache_desc {
   int32_t  batch, heads, head_dim;   /* head_dim: 64 or 128 */
   int32_t  bits;                     /* 2 or 4 */
   int32_t  group;                    /* 32, 64 or 128; divides head_dim */
-  uint32_t flags;                    /* KVQ_ROTATE_K | KVQ_ROTATE_V | KVQ_RING */
+  uint32_t flags;                    /* KVQ_ROTATE_K | KVQ_ROTATE_V | KVQ_RING | KVQ_K_PER_CHANNEL */
   int64_t  capacity;                 /* tokens per (batch, head); a multiple of 128 */
   void*    k_codes;  void* v_codes;  /* device, u8  [batch,heads,capacity, head_dim*bits/8] */
   void*    k_scale;  void* v_scale;  /* device, u8  [batch,heads,capacity, head_dim/group] (E4M3) */

@@ -22,6 +22,7 @@ KVQ_ERR_CAPACITY, KVQ_ERR_CUDA, KVQ_ERR_TIMEOUT, KVQ_ERR_WORKSPACE = -4, -5, -6,
 KVQ_ROTATE_K = 1
 KVQ_RING = 2
 KVQ_ROTATE_V = 4
+KVQ_K_PER_CHANNEL = 8
 KVQ_CORRECTION_OFF, KVQ_CORRECTION_ON, KVQ_CORRECTION_EXACT = 0, 1, 2
 KVQ_KERNEL_AUTO, KVQ_KERNEL_MMA_SYNC, KVQ_KERNEL_TCGEN05 = 0, 1 << 8, 2 << 8
 
@@ -115,10 +116,11 @@ class Cache:
     """Caller-side owner of the six device buffers of one quantized cache plus its descriptor."""
 
     def __init__(self, batch, heads, head_dim, bits, group, capacity, rotate_k=True, signs=None, device="cuda",
-                 ring=False, rotate_v=False):
+                 ring=False, rotate_v=False, k_per_channel=False):
         self.desc = kvq_cache_desc(batch, heads, head_dim, bits, group,
                                    (KVQ_ROTATE_K if rotate_k else 0) | (KVQ_RING if ring else 0)
-                                   | (KVQ_ROTATE_V if rotate_v else 0), capacity)
+                                   | (KVQ_ROTATE_V if rotate_v else 0) | (KVQ_K_PER_CHANNEL if k_per_channel else 0),
+                                   capacity)
         sizes = kvq_cache_bytes(self.desc)
         self.buffers = [torch.zeros(n, dtype=torch.uint8, device=device) for n in sizes]
         (self.desc.k_codes, self.desc.v_codes, self.desc.k_scale, self.desc.v_scale,
@@ -139,10 +141,12 @@ class Cache:
         d = self.desc
         B, H, Cp, G = d.batch, d.heads, d.capacity, self.groups
         kc, vc, ks, vs, kz, vz = self.buffers
+        # per-channel keys: one row of head_dim steps / zero-points per block of `group` tokens
+        kshape = (B, H, Cp // d.group, d.head_dim) if d.flags & KVQ_K_PER_CHANNEL else (B, H, Cp, G)
         return {
             "k_codes": kc.view(B, H, Cp, -1), "v_codes": vc.view(B, H, Cp, -1),
-            "k_scale": ks.view(B, H, Cp, G), "v_scale": vs.view(B, H, Cp, G),
-            "k_zero": kz.view(torch.int16).view(B, H, Cp, G), "v_zero": vz.view(torch.int16).view(B, H, Cp, G),
+            "k_scale": ks.view(*kshape), "v_scale": vs.view(B, H, Cp, G),
+            "k_zero": kz.view(torch.int16).view(*kshape), "v_zero": vz.view(torch.int16).view(B, H, Cp, G),
         }
 
 

@@ -30,6 +30,7 @@ struct AParams {
   const int8_t* signs;
   int64_t capacity, cache_begin;
   int heads, group, rotate, correction;   // correction: 0 off, 1 Taylor (Eq. 15), 2 exact (Eq. 12)
+  int k_per_channel;                      // App. E: key steps / zero-points per (block of `group` tokens, channel)
   int m_tokens, n_cached, n_cur;
   float scale_log2, bias_coef_log2;   // sigma*log2(e), (sigma^2/24)*log2(e)
   float softmax_scale;
@@ -113,6 +114,30 @@ __device__ __forceinline__ void dequant_store(const Packed<D, BITS>& r, uint16_t
   }
 }
 
+// Per-channel keys (App. E): x_hat = (code - zero_c) * step_c with the steps and zero-points of the key's token block,
+// staged in shared memory as floats ([D] each), rounded once to FP16.
+template <int D, int BITS>
+__device__ __forceinline__ void dequant_store_per_channel(const Packed<D, BITS>& r, uint16_t* tile, int key, int half,
+                                                          const float* step, const float* zero) {
+  constexpr int LD = D + 8;
+  constexpr int per = 32 / BITS;
+  constexpr uint32_t mask = (1u << BITS) - 1;
+  uint16_t* row = tile + key * LD + half * (D / 2);
+#pragma unroll
+  for (int c8 = 0; c8 < D / 2; c8 += 8) {
+    const int ch = half * (D / 2) + c8;
+    uint32_t o[4];
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+      const int c0 = c8 + e, c1 = c8 + e + 1;
+      const float x0 = ((float)((r.w[c0 / per] >> ((c0 % per) * BITS)) & mask) - zero[ch + e]) * step[ch + e];
+      const float x1 = ((float)((r.w[c1 / per] >> ((c1 % per) * BITS)) & mask) - zero[ch + e + 1]) * step[ch + e + 1];
+      o[e / 2] = pack_f16(x0, x1);
+    }
+    *reinterpret_cast<uint4*>(row + c8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 // log(sinh(a)/a) for a >= 0 (Eq. (12)): series below 0.5, a - log(2a) + log1p(-exp(-2a)) above.
 __device__ __forceinline__ float log_sinhc(float a) {
   if (a < 0.5f) {
@@ -139,7 +164,12 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
   // log2(e) * sum over the group's channels of log(sinh(a)/a), a = sigma |q~_c| step / 2 (Eq. (12)): a step
   // takes one of 127 values, so the exact bias of a score is one table look-up per group
   uint32_t* sWb = reinterpret_cast<uint32_t*>(sW + kBN * 4);   // [kBN]
-  float* sT = reinterpret_cast<float*>(sWb + kBN);             // [kBM][G][128]
+  // per-channel keys only: steps and zero-points of the (at most two) token blocks a 64-key tile touches, and the
+  // bias of every (query row, block): (sigma^2/24) log2(e) sum_c q~_c^2 step_c^2, one scalar for all keys of a block
+  float* sPcStep = reinterpret_cast<float*>(sWb + kBN);        // [2][D]
+  float* sPcZero = sPcStep + 2 * D;                            // [2][D]
+  float* sPcBias = sPcZero + 2 * D;                            // [kBM][2]
+  float* sT = sPcBias + kBM * 2;                               // [kBM][G][128]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.y, b = bh / p.heads, h = bh - b * p.heads;
@@ -266,6 +296,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) bsum += (j < G) ? nu[j] * sW[col * 4 + j] : 0.f;
           }
+          if (p.k_per_channel) bsum = sPcBias[((e < 2) ? rA : rB) * 2 + ((p.group == 32) ? (col >> 5) : 0)];
           v -= bsum;
         }
         if (col >= n_valid) v = -INFINITY;
@@ -324,10 +355,37 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
       const int64_t slot = p.cache_begin + min((int64_t)t * kBN + key, (int64_t)p.n_cached - 1);
       return tok_base + (slot >= p.capacity ? slot - p.capacity : slot);
     };
-    load_packed<D, BITS>(pk, p.k_codes, p.k_scale, p.k_zero, tok_of(0), half, G);
+    const int Gk = p.k_per_channel ? 0 : G;                      // per-channel keys have no per-token metadata
+    load_packed<D, BITS>(pk, p.k_codes, p.k_scale, p.k_zero, tok_of(0), half, Gk);
     load_packed<D, BITS>(pv, p.v_codes, p.v_scale, p.v_zero, tok_of(0), half, G);
     for (int t = 0; t < n_ctiles; ++t) {
       __syncthreads();
+      if (p.k_per_channel) {
+        // the tile's keys lie in one token block (group 64, 128: windows start on a block) or two (group 32)
+        const int nblk = (p.group == 32) ? 2 : 1;
+        for (int i = tid; i < nblk * D; i += kThreads) {
+          const int bi = i / D, c = i - bi * D;
+          int64_t slot = p.cache_begin + min((int64_t)t * kBN + bi * 32, (int64_t)p.n_cached - 1);
+          if (slot >= p.capacity) slot -= p.capacity;
+          const int64_t blk = (int64_t)bh * (p.capacity / p.group) + slot / p.group;
+          sPcStep[bi * D + c] = e4m3_byte_to_f32(__ldg(p.k_scale + blk * D + c));
+          sPcZero[bi * D + c] = bf16_bits_to_f32(__ldg(p.k_zero + blk * D + c));
+        }
+        __syncthreads();
+        {
+          const int r = tid >> 1, bi = tid & 1;                  // kThreads = 2 * kBM: one (row, block) per thread
+          float acc = 0.f;
+          if (p.correction && bi < nblk) {
+            for (int c = 0; c < D; ++c) {
+              const float qv = __half2float(__ushort_as_half(sQr[r * LD + c])), ds = sPcStep[bi * D + c];
+              acc += qv * qv * ds * ds;
+            }
+          }
+          sPcBias[r * 2 + bi] = p.bias_coef_log2 * acc;
+        }
+        dequant_store_per_channel<D, BITS>(pk, sK, key, half, sPcStep + ((p.group == 32) ? (key >> 5) : 0) * D,
+                                           sPcZero + ((p.group == 32) ? (key >> 5) : 0) * D);
+      } else
       dequant_store<D, BITS, true>(pk, sK, key, half, p.group);
       dequant_store<D, BITS, false>(pv, sV, key, half, p.group);
       if (half == 0) {
@@ -340,7 +398,7 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
       }
       __syncthreads();
       if (t + 1 < n_ctiles) {
-        load_packed<D, BITS>(pk, p.k_codes, p.k_scale, p.k_zero, tok_of(t + 1), half, G);
+        load_packed<D, BITS>(pk, p.k_codes, p.k_scale, p.k_zero, tok_of(t + 1), half, Gk);
         load_packed<D, BITS>(pv, p.v_codes, p.v_scale, p.v_zero, tok_of(t + 1), half, G);
       }
       process_tile(min(kBN, p.n_cached - t * kBN), true);
@@ -405,7 +463,8 @@ __global__ void __launch_bounds__(kThreads) attn_mma_sync_kernel(AParams p) {
 template <int D, int BITS>
 int launch(const AParams& p, dim3 grid, cudaStream_t st) {
   constexpr int LD = D + 8;
-  constexpr size_t base = (size_t)(2 * kBM + 2 * kBN) * LD * 2 + (kBM + kBN) * 4 * sizeof(float) + kBN * sizeof(uint32_t);
+  constexpr size_t base = (size_t)(2 * kBM + 2 * kBN) * LD * 2 + (kBM + kBN) * 4 * sizeof(float) + kBN * sizeof(uint32_t) +
+                          (size_t)(4 * D + 2 * kBM) * sizeof(float);
   // the exact correction adds its table: 64 rows x groups x 128 step values
   const size_t smem = base + (p.correction == 2 ? (size_t)kBM * (D / p.group) * 128 * sizeof(float) : 0);
   static bool configured = false;
@@ -438,6 +497,7 @@ int launch_attn_mma_sync(const AttnArgs& a) {
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
   p.correction = (a.flags & KVQ_CORRECTION_EXACT) ? 2 : ((a.flags & KVQ_CORRECTION_ON) ? 1 : 0);
   p.softmax_scale = a.softmax_scale;
+  p.k_per_channel = (d->flags & KVQ_K_PER_CHANNEL) ? 1 : 0;
   p.m_tokens = (int)a.m_tokens; p.n_cached = (int)a.cache_len; p.n_cur = (int)a.n_cur;
   p.scale_log2 = a.softmax_scale * kLog2e;
   p.bias_coef_log2 = a.softmax_scale * a.softmax_scale / 24.0f * kLog2e;

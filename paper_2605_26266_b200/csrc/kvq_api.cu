@@ -19,7 +19,7 @@ int check_shape(const kvq_cache_desc* d) {
   if (d->bits != 2 && d->bits != 4) return KVQ_ERR_UNSUPPORTED;
   if (d->group != 32 && d->group != 64 && d->group != 128) return KVQ_ERR_UNSUPPORTED;
   if (d->capacity % 128 != 0) return KVQ_ERR_INVALID_ARG;
-  if (d->flags & ~(KVQ_ROTATE_K | KVQ_ROTATE_V | KVQ_RING)) return KVQ_ERR_INVALID_ARG;
+  if (d->flags & ~(KVQ_ROTATE_K | KVQ_ROTATE_V | KVQ_RING | KVQ_K_PER_CHANNEL)) return KVQ_ERR_INVALID_ARG;
   return KVQ_OK;
 }
 
@@ -48,6 +48,8 @@ static int check_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t
   if (r != KVQ_OK) return r;
   if (cache_begin < 0 || cache_len < 0 || m_tokens < 0 || n_cur < 1) return KVQ_ERR_INVALID_ARG;
   if (cache_begin % 16 != 0) return KVQ_ERR_ALIGNMENT;
+  if ((d->flags & KVQ_K_PER_CHANNEL) && cache_begin % d->group != 0) return KVQ_ERR_ALIGNMENT;   // windows start on a block
+  if ((d->flags & KVQ_K_PER_CHANNEL) && (flags & KVQ_CORRECTION_EXACT)) return KVQ_ERR_UNSUPPORTED;
   // linear cache: the window ends inside the capacity; ring cache: it has at most `capacity` tokens
   if (((d->flags & KVQ_RING) ? cache_len : cache_begin + cache_len) > d->capacity) return KVQ_ERR_CAPACITY;
   if (m_tokens > 0x7FFFFFFFLL || n_cur > 0x7FFFFFFFLL || cache_len > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
@@ -72,7 +74,7 @@ static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur
   *err = KVQ_OK;
   if (kern == KVQ_KERNEL_MMA_SYNC) return false;
   // the exact correction (a table look-up per score and group) exists in the warp-level kernel only
-  const bool ok = attn_tcgen05_supports(d, m_tokens, n_cur) && !(flags & KVQ_CORRECTION_EXACT);
+  const bool ok = attn_tcgen05_supports(d, m_tokens, n_cur) && !(flags & KVQ_CORRECTION_EXACT) && !(d->flags & KVQ_K_PER_CHANNEL);
   if (kern == KVQ_KERNEL_TCGEN05 && !ok) *err = KVQ_ERR_UNSUPPORTED;
   return ok;
 }
@@ -119,6 +121,8 @@ int kvq_quantize_append(const kvq_cache_desc* desc, int64_t cache_len, const voi
   if (r != KVQ_OK) return r;
   if (cache_len < 0 || n_tokens < 0) return KVQ_ERR_INVALID_ARG;
   if (((desc->flags & KVQ_RING) ? n_tokens : cache_len + n_tokens) > desc->capacity) return KVQ_ERR_CAPACITY;
+  if ((desc->flags & KVQ_K_PER_CHANNEL) && (cache_len % desc->group != 0 || n_tokens % desc->group != 0))
+    return KVQ_ERR_ALIGNMENT;                          // per-channel keys come in whole blocks of `group` tokens
   if ((r = check_tensor(k_bf16, kv)) != KVQ_OK) return r;
   if ((r = check_tensor(v_bf16, kv)) != KVQ_OK) return r;
   if (n_tokens == 0) return KVQ_OK;
@@ -209,7 +213,8 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
   if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
   if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
   if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
-  if (!attn_tcgen05_supports(desc, m_tokens, n_cur) || (flags & KVQ_CORRECTION_EXACT) || (desc->flags & KVQ_ROTATE_V))
+  if (!attn_tcgen05_supports(desc, m_tokens, n_cur) || (flags & KVQ_CORRECTION_EXACT) ||
+      (desc->flags & (KVQ_ROTATE_V | KVQ_K_PER_CHANNEL)))
     return KVQ_ERR_UNSUPPORTED;
   if (m_tokens == 0) return KVQ_OK;
   AttnArgs a;

@@ -25,6 +25,7 @@ struct QParams {
   int64_t sb, sh, st;          // element strides of k and v
   int64_t n_tokens, cache_len, capacity;
   int heads, group, rotate, rotate_v;
+  int skip_k;                  // per-channel keys: the keys are written by quantize_k_per_channel_kernel instead
   const int8_t* signs;
   uint8_t* codes[2]; uint8_t* scale[2]; uint16_t* zero[2];
   int tiles_per_bh;
@@ -230,14 +231,16 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
     decode_vec<EPL>(rk, x);
     const RawVec<EPL> rv_cur = rv;
     if (tile_g + (int)gridDim.x < total_tiles) fetch(tile_g + (int)gridDim.x);
-    if (p.rotate) {
-      if (p.signs) {
+    if (!p.skip_k) {
+      if (p.rotate) {
+        if (p.signs) {
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], (float)p.signs[l8 * EPL + e]);
+          for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], (float)p.signs[l8 * EPL + e]);
+        }
+        hadamard<EPL>(x, l8, c_d);
       }
-      hadamard<EPL>(x, l8, c_d);
+      quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[0], s_scale[0], s_zero[0]);
     }
-    quantize_stage<EPL, BITS, GROUP>(x, l8, tok, s_codes[0], s_scale[0], s_zero[0]);
     decode_vec<EPL>(rv_cur, x);
     if (p.rotate_v) {                                       // values stored rotated too (KVQ_ROTATE_V)
       if (p.signs) {
@@ -261,6 +264,7 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
       const int64_t tok_index = (int64_t)bh * p.capacity + (piece ? 0 : slot0);
 #pragma unroll
       for (int w = 0; w < 2; ++w) {
+        if (w == 0 && p.skip_k) continue;
         copy_out(p.codes[w] + tok_index * CB, reinterpret_cast<const uint8_t*>(s_codes[w]) + skip * CB, ntok * CB, threadIdx.x, kWarps * 32);
         copy_out(p.scale[w] + tok_index * G, s_scale[w] + skip * G, ntok * G, threadIdx.x, kWarps * 32);
         copy_out(reinterpret_cast<uint8_t*>(p.zero[w] + tok_index * G), reinterpret_cast<const uint8_t*>(s_zero[w] + skip * G),
@@ -268,6 +272,75 @@ __global__ void __launch_bounds__(kWarps * 32) quantize_append_kernel(QParams p)
       }
     }
     __syncthreads();
+  }
+}
+
+// ---- per-channel keys (App. E) -----------------------------------------------------------------------
+// One CTA per (batch*head, block of g = p.group tokens): the g x D block is rotated into shared memory (FP32), then
+// thread c owns channel c: minimum and maximum over the block's tokens, step and zero-point with the arithmetic of
+// Eq. (1) in plain IEEE operations (range / L, E4M3 rounding, -rint(min / step), rint(y / step) + zero, clamp),
+// codes as bytes in shared memory; finally the codes of a token are packed 32 / BITS per word along the channels,
+// the layout every other kernel reads.  An analysis option: nothing here is tuned.
+template <int D, int BITS>
+__global__ void __launch_bounds__(256) quantize_k_per_channel_kernel(QParams p) {
+  constexpr int EPL = D / 8;
+  constexpr int CB = D * BITS / 8;
+  constexpr int LDY = D + 1;
+  extern __shared__ __align__(16) uint8_t pc_smem[];
+  const int g = p.group;
+  float* y = reinterpret_cast<float*>(pc_smem);                       // [g][D + 1]
+  uint8_t* codes = pc_smem + (size_t)g * LDY * sizeof(float);          // [g][D]
+  const int bh = blockIdx.y, b = bh / p.heads, h = bh - b * p.heads;
+  const int64_t t0 = (int64_t)blockIdx.x * g;                          // first token of the block within the chunk
+  const int lane = threadIdx.x & 31, l8 = lane & 7;
+  const float c_d = (D == 64) ? 0.125f : __uint_as_float(0x3DB504F3u);
+  for (int r = threadIdx.x >> 3; r < g; r += 32) {                     // 8 lanes per token, 32 tokens per pass
+    RawVec<EPL> raw;
+    load_raw_vec<EPL>(raw, p.k + (int64_t)b * p.sb + (int64_t)h * p.sh + (t0 + r) * p.st, l8);
+    float x[EPL];
+    decode_vec<EPL>(raw, x);
+    if (p.rotate) {
+      if (p.signs) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) x[e] = __fmul_rn(x[e], (float)p.signs[l8 * EPL + e]);
+      }
+      hadamard<EPL>(x, l8, c_d);
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) y[r * LDY + l8 * EPL + e] = x[e];
+  }
+  __syncthreads();
+  int64_t slot0 = p.cache_len + t0;                                    // whole blocks never straddle the end of a ring
+  slot0 %= p.capacity;
+  if (threadIdx.x < D) {
+    const int c = threadIdx.x;
+    constexpr float L = (float)((1 << BITS) - 1);
+    float mn = y[c], mx = y[c];
+    for (int t = 1; t < g; ++t) { mn = fminf(mn, y[t * LDY + c]); mx = fmaxf(mx, y[t * LDY + c]); }
+    const float step = __fdiv_rn(__fsub_rn(mx, mn), L);
+    uint32_t sbyte = f32_to_e4m3_byte(step);
+    if (sbyte == 0) sbyte = 1;                                         // floor at the smallest subnormal 2^-9
+    const float ds = e4m3_byte_to_f32(sbyte);
+    const float z = __fsub_rn(0.0f, rintf(__fdiv_rn(mn, ds)));
+    const uint32_t zbits = f32_to_bf16_bits(z);
+    const float zs = bf16_bits_to_f32(zbits);
+    for (int t = 0; t < g; ++t) {
+      const float cc = fminf(fmaxf(__fadd_rn(rintf(__fdiv_rn(y[t * LDY + c], ds)), zs), 0.0f), L);
+      codes[t * D + c] = (uint8_t)cc;
+    }
+    const int64_t blk = (int64_t)bh * (p.capacity / g) + slot0 / g;
+    p.scale[0][blk * D + c] = (uint8_t)sbyte;
+    p.zero[0][blk * D + c] = (uint16_t)zbits;
+  }
+  __syncthreads();
+  constexpr int kPer = 32 / BITS;                                      // codes per 32-bit word
+  uint32_t* out = reinterpret_cast<uint32_t*>(p.codes[0] + ((int64_t)bh * p.capacity + slot0) * CB);
+  for (int i = threadIdx.x; i < g * (CB / 4); i += 256) {
+    const int t = i / (CB / 4), w = i - t * (CB / 4);
+    uint32_t word = 0;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) word |= (uint32_t)codes[t * D + w * kPer + j] << (j * BITS);
+    out[i] = word;                                                     // tokens of a block are contiguous: out[t * CB/4 + w]
   }
 }
 
@@ -297,6 +370,7 @@ int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const voi
   p.n_tokens = n_tokens; p.cache_len = cache_len % d->capacity; p.capacity = d->capacity;
   p.heads = d->heads; p.group = d->group; p.rotate = (d->flags & KVQ_ROTATE_K) ? 1 : 0;
   p.rotate_v = (d->flags & KVQ_ROTATE_V) ? 1 : 0;
+  p.skip_k = (d->flags & KVQ_K_PER_CHANNEL) ? 1 : 0;
   p.signs = d->signs;
   p.codes[0] = static_cast<uint8_t*>(d->k_codes); p.codes[1] = static_cast<uint8_t*>(d->v_codes);
   p.scale[0] = static_cast<uint8_t*>(d->k_scale); p.scale[1] = static_cast<uint8_t*>(d->v_scale);
@@ -319,6 +393,18 @@ int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const voi
 #undef KVQ_QA
   if (!launched) return KVQ_ERR_UNSUPPORTED;
   KVQ_CUDA_TRY(cudaGetLastError());
+  if (p.skip_k) {                                     // per-channel keys: one CTA per block of `group` tokens
+    const int64_t bh = (int64_t)d->batch * d->heads;
+    if (bh > 65535) return KVQ_ERR_UNSUPPORTED;
+    const dim3 pgrid((unsigned)(n_tokens / d->group), (unsigned)bh);
+    const size_t smem = (size_t)d->group * (d->head_dim + 1) * sizeof(float) + (size_t)d->group * d->head_dim;
+#define KVQ_PC(D_, B_) if (d->head_dim == D_ && d->bits == B_) { \
+      KVQ_CUDA_TRY(cudaFuncSetAttribute(quantize_k_per_channel_kernel<D_, B_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+      quantize_k_per_channel_kernel<D_, B_><<<pgrid, 256, smem, st>>>(p); }
+    KVQ_PC(128, 2) KVQ_PC(128, 4) KVQ_PC(64, 2) KVQ_PC(64, 4)
+#undef KVQ_PC
+    KVQ_CUDA_TRY(cudaGetLastError());
+  }
   return KVQ_OK;
 }
 

@@ -99,6 +99,6 @@ def test_ring_cache_argument_rules_without_gpu(binding):
     assert args(1024, 257, 0) == b.KVQ_ERR_CAPACITY
     assert args(1000, 16, 0) == b.KVQ_ERR_ALIGNMENT
     assert b.lib.kvq_unpack_codes(C.byref(ring), 0, 250, 257, 0x1000, None) == b.KVQ_ERR_CAPACITY
-    unknown = b.kvq_cache_desc(1, 2, 128, 2, 32, 8, 256)
+    unknown = b.kvq_cache_desc(1, 2, 128, 2, 32, 16, 256)
     sizes = (C.c_size_t * 6)()
     assert b.lib.kvq_cache_bytes(C.byref(unknown), sizes) == b.KVQ_ERR_INVALID_ARG
