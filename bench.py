@@ -242,6 +242,36 @@ def main():
     step_ms = float((attn_ms + app_ms).mean())
     if int(status.item()) != 0:
         raise SystemExit(f"device-side wait timed out, status {int(status.item())}")
+    eager_step_ms = step_ms
+
+    # The step's kernels replayed from a CUDA graph (the calls only enqueue on the caller's stream, so they
+    # capture as they are): the same work without the gaps between launches.  `value` is taken from this run,
+    # the per-kernel times above from the eager one.
+    if not args.profile:
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                B.kvq_attn_corrected(cache, q, k, v, sigma, flags, cache_len=n_cached, out=out, status_word=status)
+                B.kvq_quantize_append(cache, k, v, cache_len=n_cached)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            flush.zero_()
+            graph.replay()
+        grecs = []
+        barrier()
+        for _ in range(args.steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            grecs.append((e0, e1))
+        barrier()
+        step_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in grecs]))
+        if int(status.item()) != 0:
+            raise SystemExit(f"device-side wait timed out, status {int(status.item())}")
 
     # correction off, same kernel: cost of the correction
     recs_off = []
@@ -320,8 +350,9 @@ def main():
         e2e_ms = pipelined(n_e2e)
         barrier()
     # ---- reduce over ranks: slowest rank's time ----
-    step_ms, attn_mean, app_mean, attn_off_ms, e2e_ms = replicas.max_over_ranks(
-        [step_ms, float(attn_ms.mean()), float(app_ms.mean()), attn_off_ms, 0.0 if args.no_e2e else e2e_ms], device=dev)
+    step_ms, attn_mean, app_mean, attn_off_ms, e2e_ms, eager_step_ms = replicas.max_over_ranks(
+        [step_ms, float(attn_ms.mean()), float(app_ms.mean()), attn_off_ms, 0.0 if args.no_e2e else e2e_ms,
+         eager_step_ms], device=dev)
 
     if rank == 0:
         flops = w.flops()
@@ -333,6 +364,8 @@ def main():
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
+            "launch": "eager calls (--profile)" if args.profile else "step replayed from a CUDA graph",
+            "ms_per_step_eager": eager_step_ms,
             "us_per_call": {"attn_corrected": attn_mean * 1e3, "attn_uncorrected": attn_off_ms * 1e3,
                             "quantize_append": app_mean * 1e3,
                             "correction_overhead": attn_mean / attn_off_ms - 1.0},
