@@ -79,6 +79,36 @@ static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur
   return ok;
 }
 
+// Checks shared by the two attention entry points, then the argument block the launchers take.
+static int check_attn_call(const kvq_cache_desc* d, int64_t cache_begin, int64_t cache_len, const void* q,
+                           kvq_strides qs, const void* k_cur, const void* v_cur, kvq_strides kvs, int64_t m_tokens,
+                           int64_t n_cur, const void* out, kvq_strides os, float softmax_scale, uint32_t flags) {
+  int r = check_attn_args(d, cache_begin, cache_len, m_tokens, n_cur, flags);
+  if (r != KVQ_OK) return r;
+  if ((r = check_desc(d)) != KVQ_OK) return r;
+  if ((r = check_tensor(q, qs)) != KVQ_OK) return r;
+  if ((r = check_tensor(k_cur, kvs)) != KVQ_OK) return r;
+  if ((r = check_tensor(v_cur, kvs)) != KVQ_OK) return r;
+  if ((r = check_tensor(out, os)) != KVQ_OK) return r;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
+  return KVQ_OK;
+}
+
+static AttnArgs make_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t cache_len, const void* q,
+                               kvq_strides qs, const void* k_cur, const void* v_cur, kvq_strides kvs,
+                               int64_t m_tokens, int64_t n_cur, void* out, kvq_strides os, float softmax_scale,
+                               uint32_t flags, float* lse, float* cached_mass, void* workspace,
+                               size_t workspace_bytes, int32_t* status_word, kvq_stream_t stream) {
+  AttnArgs a;
+  a.desc = d; a.cache_begin = cache_begin; a.cache_len = cache_len;
+  a.q = q; a.qs = qs; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kvs; a.vs = kvs;
+  a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out; a.os = os;
+  a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse; a.cached_mass = cached_mass;
+  a.workspace = workspace; a.workspace_bytes = workspace_bytes; a.status_word = status_word;
+  a.stream = (cudaStream_t)stream;
+  return a;
+}
+
 }  // namespace kvq
 
 using namespace kvq;
@@ -160,14 +190,9 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
                        kvq_strides o_strides, float softmax_scale, uint32_t flags, float* lse_out,
                        float* cached_mass_out, void* workspace, size_t workspace_bytes,
                        int32_t* status_word, kvq_stream_t stream) {
-  int r = check_attn_args(desc, cache_begin, cache_len, m_tokens, n_cur, flags);
+  int r = check_attn_call(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens, n_cur,
+                          out_bf16, o_strides, softmax_scale, flags);
   if (r != KVQ_OK) return r;
-  if ((r = check_desc(desc)) != KVQ_OK) return r;
-  if ((r = check_tensor(q, q_strides)) != KVQ_OK) return r;
-  if ((r = check_tensor(k_cur, kv_strides)) != KVQ_OK) return r;
-  if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
-  if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
-  if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
@@ -180,13 +205,9 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
     }
   }
   if (m_tokens == 0) return KVQ_OK;
-  AttnArgs a;
-  a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;
-  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides; a.vs = kv_strides;
-  a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out_bf16; a.os = o_strides;
-  a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse_out; a.cached_mass = cached_mass_out;
-  a.workspace = workspace; a.workspace_bytes = workspace_bytes; a.status_word = status_word;
-  a.stream = (cudaStream_t)stream;
+  AttnArgs a = make_attn_args(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens, n_cur,
+                              out_bf16, o_strides, softmax_scale, flags, lse_out, cached_mass_out, workspace,
+                              workspace_bytes, status_word, stream);
   if (rotv) {
     // values are cached rotated: bring the current chunk's values into the same space, attend, rotate the output back
     const kvq_strides dense{(int64_t)desc->heads * n_cur * desc->head_dim, n_cur * (int64_t)desc->head_dim, (int64_t)desc->head_dim};
@@ -205,25 +226,16 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
                                       kvq_strides o_strides, float softmax_scale, uint32_t flags, float* lse_out,
                                       float* cached_mass_out, int32_t* status_word, kvq_stream_t stream) {
   if (flags & KVQ_KERNEL_MASK) return KVQ_ERR_INVALID_ARG;      // this entry point has one kernel only
-  int r = check_attn_args(desc, cache_begin, cache_len, m_tokens, n_cur, flags);
+  int r = check_attn_call(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens, n_cur,
+                          out_bf16, o_strides, softmax_scale, flags);
   if (r != KVQ_OK) return r;
-  if ((r = check_desc(desc)) != KVQ_OK) return r;
-  if ((r = check_tensor(q, q_strides)) != KVQ_OK) return r;
-  if ((r = check_tensor(k_cur, kv_strides)) != KVQ_OK) return r;
-  if ((r = check_tensor(v_cur, kv_strides)) != KVQ_OK) return r;
-  if ((r = check_tensor(out_bf16, o_strides)) != KVQ_OK) return r;
-  if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
   if (!attn_tcgen05_supports(desc, m_tokens, n_cur) || (flags & KVQ_CORRECTION_EXACT) ||
       (desc->flags & (KVQ_ROTATE_V | KVQ_K_PER_CHANNEL)))
     return KVQ_ERR_UNSUPPORTED;
   if (m_tokens == 0) return KVQ_OK;
-  AttnArgs a;
-  a.desc = desc; a.cache_begin = cache_begin; a.cache_len = cache_len;
-  a.q = q; a.qs = q_strides; a.k_cur = k_cur; a.v_cur = v_cur; a.kvs = kv_strides; a.vs = kv_strides;
-  a.m_tokens = m_tokens; a.n_cur = n_cur; a.out = out_bf16; a.os = o_strides;
-  a.softmax_scale = softmax_scale; a.flags = flags; a.lse = lse_out; a.cached_mass = cached_mass_out;
-  a.workspace = nullptr; a.workspace_bytes = 0; a.status_word = status_word;
-  a.stream = (cudaStream_t)stream;
+  const AttnArgs a = make_attn_args(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens,
+                                    n_cur, out_bf16, o_strides, softmax_scale, flags, lse_out, cached_mass_out,
+                                    nullptr, 0, status_word, stream);
   return launch_attn_tcgen05_static(a);
 }
 
