@@ -58,6 +58,15 @@ def test_error_bound_and_clamping():
             yg = y.reshape(2000, 128 // group, group)
             exact = (yg.max(-1) - yg.min(-1)) / L
             assert np.all(np.abs(O.e4m3_decode(sb) - exact) <= np.maximum(exact / 16, 2.0 ** -10) * (1 + 1e-6))
+            # the step and the zero-point cover [min, max] (the sentence below Eq. (1)): with the zero-point taken
+            # from the stored step, the minimum of a group gets code 0 exactly, and the maximum, whose distance
+            # from it is at least L / (1 + 2^-4) stored steps, code L - 1 or L
+            cg = codes.reshape(2000, 128 // group, group)
+            at_min = np.take_along_axis(cg, yg.argmin(-1)[..., None], -1)[..., 0]
+            at_max = np.take_along_axis(cg, yg.argmax(-1)[..., None], -1)[..., 0]
+            normal = O.e4m3_decode(sb) >= 2.0 ** -6
+            assert np.all(at_min[normal] == 0)
+            assert np.all(at_max[normal] >= L - 1)
 
 
 def _scalar_quantize_f32(vec, bits, group):
