@@ -47,7 +47,7 @@ extern "C" {
 /* status codes */
 #define KVQ_OK                 0
 #define KVQ_ERR_INVALID_ARG   -1   /* null pointer, non-positive size, group does not divide head_dim */
-#define KVQ_ERR_UNSUPPORTED   -2   /* head_dim / bits / group combination not built */
+#define KVQ_ERR_UNSUPPORTED   -2   /* head_dim / bits / group combination not built, or batch * heads > 65535 */
 #define KVQ_ERR_ALIGNMENT     -3   /* pointer not 16-byte aligned, stride not a multiple of 8 elements */
 #define KVQ_ERR_CAPACITY      -4   /* the append or the window would run past `capacity` */
 #define KVQ_ERR_CUDA          -5   /* a CUDA runtime/driver call failed; see kvq_last_cuda_error() */
@@ -89,7 +89,7 @@ typedef void* kvq_stream_t;          /* a cudaStream_t */
 
 /* Describes one caller-owned cache.  Plain data, host memory. */
 typedef struct kvq_cache_desc {
-  int32_t  batch, heads, head_dim;   /* head_dim: 64 or 128 */
+  int32_t  batch, heads, head_dim;   /* head_dim: 64 or 128; batch * heads <= 65535 (a grid dimension) */
   int32_t  bits;                     /* 2 or 4 */
   int32_t  group;                    /* 32, 64 or 128; divides head_dim */
   uint32_t flags;                    /* KVQ_ROTATE_K | KVQ_ROTATE_V | KVQ_RING | KVQ_K_PER_CHANNEL */

@@ -16,6 +16,7 @@ int check_shape(const kvq_cache_desc* d) {
     return KVQ_ERR_INVALID_ARG;
   if (d->head_dim % d->group != 0) return KVQ_ERR_INVALID_ARG;
   if (d->head_dim != 64 && d->head_dim != 128) return KVQ_ERR_UNSUPPORTED;
+  if ((int64_t)d->batch * d->heads > 65535) return KVQ_ERR_UNSUPPORTED;     // (batch, head) is a grid dimension
   if (d->bits != 2 && d->bits != 4) return KVQ_ERR_UNSUPPORTED;
   if (d->group != 32 && d->group != 64 && d->group != 128) return KVQ_ERR_UNSUPPORTED;
   if (d->capacity % 128 != 0) return KVQ_ERR_INVALID_ARG;

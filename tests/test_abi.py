@@ -56,6 +56,10 @@ def test_argument_errors_without_gpu(binding):
     assert b.lib.kvq_cache_bytes(C.byref(bad), sizes) == b.KVQ_ERR_INVALID_ARG
     bad = b.kvq_cache_desc(1, 2, 128, 3, 32, 0, 128)
     assert b.lib.kvq_cache_bytes(C.byref(bad), sizes) == b.KVQ_ERR_UNSUPPORTED
+    bad = b.kvq_cache_desc(2048, 32, 128, 2, 32, 0, 128)        # batch * heads is a grid dimension: at most 65535
+    assert b.lib.kvq_cache_bytes(C.byref(bad), sizes) == b.KVQ_ERR_UNSUPPORTED
+    ok = b.kvq_cache_desc(2047, 32, 128, 2, 32, 0, 128)
+    assert b.lib.kvq_cache_bytes(C.byref(ok), sizes) == b.KVQ_OK
     bad = b.kvq_cache_desc(1, 2, 128, 2, 32, 0, 100)
     assert b.lib.kvq_cache_bytes(C.byref(bad), sizes) == b.KVQ_ERR_INVALID_ARG
     assert b.lib.kvq_cache_bytes(None, sizes) == b.KVQ_ERR_INVALID_ARG
