@@ -96,8 +96,11 @@ struct TParams {
   const uint16_t* ax_rows; // workspace: bias operand rows written by rotate_query_kernel, [batch*heads][m_tokens][8]
 };
 
-// One partial result: the segment's own normalised output O / l as BF16 [256][128], then FP32 m[256],
-// l_cur[256], l_cached[256] (running maximum in log2 units and the row sums over current and cached keys).
+// One partial result: the segment's own normalised output O / l as BF16, then FP32 m[256], l_cur[256],
+// l_cached[256] (running maximum in log2 units and the row sums over current and cached keys).  The output is
+// stored by 16-byte pieces of 8 columns, piece (column group g, row r) at (g * 256 + r) * 16: the softmax
+// threads hold one row each, so the 32 lanes of a store instruction write 512 contiguous bytes (row-major, they
+// would write 32 pieces 256 bytes apart, and the load/store unit takes them one line at a time).
 constexpr int kSlotStats = 256 * kD * 2;
 constexpr int kSlotBytes = kSlotStats + 3 * 256 * 4;
 static_assert(kSlotBytes % 256 == 0, "slots stay 256-byte aligned");
@@ -802,8 +805,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const float l = lc + la;
         const float inv = 1.0f / l;
         if (!whole || row < p.m_tokens) {
-          uint16_t* dst = whole ? p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + half * 64
-                                : reinterpret_cast<uint16_t*>(slot) + r256 * kD + half * 64;
+          // consecutive 8-column pieces: 16 bytes apart in a row of the output, 4096 bytes apart in a slot
+          uint8_t* dst = whole ? reinterpret_cast<uint8_t*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + half * 64)
+                               : slot + ((half * 8) * 256 + r256) * 16;
+          const int piece = whole ? 16 : 4096;
 #pragma unroll
           for (int i = 0; i < 64; i += 8) {
             uint4 v;
@@ -811,7 +816,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             v.y = cvt_bf16x2(__uint_as_float(sr[i + 2]) * inv, __uint_as_float(sr[i + 3]) * inv);
             v.z = cvt_bf16x2(__uint_as_float(sr[i + 4]) * inv, __uint_as_float(sr[i + 5]) * inv);
             v.w = cvt_bf16x2(__uint_as_float(sr[i + 6]) * inv, __uint_as_float(sr[i + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + i) = v;
+            *reinterpret_cast<uint4*>(dst + (i >> 3) * piece) = v;
           }
           if (half == 0) {
             if (whole) {
@@ -943,13 +948,17 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
   __syncthreads();
   const int c_first = s_first, c_last = s_last, first_slot = s_first_slot;
   if (c_first == c_last) return;                       // the unit was computed whole by one CTA
-  const int cg = threadIdx.x & 15;
+  // A thread combines the 8-column piece (cg, row): consecutive lanes take consecutive rows, which are 16 bytes
+  // apart in a slot.  The finished pieces change places through shared memory so that the output rows are
+  // written 256 contiguous bytes at a time.
+  __shared__ uint4 s_tile[16 * 16];
+  const int cg = threadIdx.x >> 4, rr = threadIdx.x & 15;
   const int bh = unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
 #pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
-  const int r256 = blockIdx.y * 64 + pass * 16 + (threadIdx.x >> 4);
+  const int r256 = blockIdx.y * 64 + pass * 16 + rr;
   const int row = (unit - bh * p.q_blocks) * 256 + r256;
-  if (row >= p.m_tokens) break;
+  if ((unit - bh * p.q_blocks) * 256 + blockIdx.y * 64 + pass * 16 >= p.m_tokens) break;     // same for the whole block
   // Partials are taken four at a time with all of their loads issued before any is used: a thread moves only
   // 16 bytes per partial, so the kernel lives on loads in flight.
   auto slot_of = [&](int c) { return p.partial + (size_t)(2 * c + (c == c_first ? first_slot : 0)) * kSlotBytes; };
@@ -974,7 +983,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
       const float* st = reinterpret_cast<const float*>(sl + kSlotStats);
       sm[j] = have ? st[r256] : -INFINITY;                  // weight 2^(-inf) = 0 for the slots that are not there
       sc[j] = st[256 + r256]; sa[j] = st[512 + r256];
-      a[j] = *reinterpret_cast<const uint4*>(sl + ((size_t)r256 * kD + cg * 8) * 2);
+      a[j] = *reinterpret_cast<const uint4*>(sl + ((size_t)cg * 256 + r256) * 16);
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -992,8 +1001,16 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
   uint4 v;
   v.x = cvt_bf16x2(acc[0] * inv, acc[1] * inv); v.y = cvt_bf16x2(acc[2] * inv, acc[3] * inv);
   v.z = cvt_bf16x2(acc[4] * inv, acc[5] * inv); v.w = cvt_bf16x2(acc[6] * inv, acc[7] * inv);
-  *reinterpret_cast<uint4*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + cg * 8) = v;
-  if (cg == 0) {
+  s_tile[rr * 16 + (cg ^ rr)] = v;
+  __syncthreads();
+  {
+    const int orr = threadIdx.x >> 4, ocg = threadIdx.x & 15;          // output side: a row per 16 lanes
+    const int orow = row - rr + orr;
+    if (orow < p.m_tokens)
+      *reinterpret_cast<uint4*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)orow * p.o_st + ocg * 8) = s_tile[orr * 16 + (ocg ^ orr)];
+  }
+  __syncthreads();
+  if (cg == 0 && row < p.m_tokens) {
     const int64_t idx = (int64_t)bh * p.m_tokens + row;
     if (p.lse) p.lse[idx] = (m + log2f(l)) * 0.6931471805599453f;
     if (p.cached_mass) p.cached_mass[idx] = l_cac * inv;
