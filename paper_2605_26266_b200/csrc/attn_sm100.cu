@@ -522,7 +522,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       while (ok && sch.next(sg)) {
         const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
         const int row0 = (sg.unit - bh * p.q_blocks) * (2 * kBlockM);
-        // the query buffer is free once every score MMA of the previous segment has retired
+        // the query buffer is free once every score MMA of the previous segment has retired (the MMA warp says so
+        // in its last iteration, before the last P V products)
         if (!(ok = cx.wait(kQEmpty, (nseg & 1) ^ 1, 100))) break;
         // a segment that starts in the cache never needs the unrotated query: load the rotated one right away
         const bool cached0 = sg.tb >= n_rt;
@@ -649,6 +650,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const int s = it & 1, s1 = (it + 1) & 1;
           const uint32_t ph = (it >> 1) & 1, ph1 = ((it + 1) >> 1) & 1;
           if (rot && !has_pv) commit1(cx.bar(kQCurDone));        // the segment starts in the cache
+          // last iteration: every score MMA of the segment is issued, so the query buffer (and the bias rows) can
+          // be handed to the next segment while the last P V products still run
+          if (!has_qk) commit1(cx.bar(kQEmpty));
 #pragma unroll 1
           for (int step = 0; step < 4; ++step) {
             const int op = rot ? step : (((step & 1) << 1) | (step >> 1));   // bit 1: scores, bit 0: query tile
@@ -678,7 +682,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         if (!ok) break;
-        commit1(cx.bar(kQEmpty));
         ++nseg;
       }
       // everything issued so far must have retired before TMEM is freed
