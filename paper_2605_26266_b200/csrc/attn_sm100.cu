@@ -924,7 +924,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 }
 
 // Combines the partial results of every unit whose key tiles were split over several CTAs.
-// grid (n_units - n_whole, 4): a block handles 64 rows x 128 columns, 16 rows at a time; thread = (row, 8-column group).
+// grid (n_units - n_whole, 16): a block handles 16 rows x 128 columns; thread = (8-column piece, row).
 __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_ctas) {
   const int unit = p.n_whole + blockIdx.x;
   const int T = p.tiles;
@@ -957,11 +957,9 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
   __shared__ uint4 s_tile[16 * 16];
   const int cg = threadIdx.x >> 4, rr = threadIdx.x & 15;
   const int bh = unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
-#pragma unroll 1
-  for (int pass = 0; pass < 4; ++pass) {
-  const int r256 = blockIdx.y * 64 + pass * 16 + rr;
+  const int r256 = blockIdx.y * 16 + rr;
   const int row = (unit - bh * p.q_blocks) * 256 + r256;
-  if ((unit - bh * p.q_blocks) * 256 + blockIdx.y * 64 + pass * 16 >= p.m_tokens) break;     // same for the whole block
+  if (row - rr >= p.m_tokens) return;                  // the same for the whole block: no rows left in this block
   // Partials are taken four at a time with all of their loads issued before any is used: a thread moves only
   // 16 bytes per partial, so the kernel lives on loads in flight.
   auto slot_of = [&](int c) { return p.partial + (size_t)(2 * c + (c == c_first ? first_slot : 0)) * kSlotBytes; };
@@ -1012,12 +1010,10 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
     if (orow < p.m_tokens)
       *reinterpret_cast<uint4*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)orow * p.o_st + ocg * 8) = s_tile[orr * 16 + (ocg ^ orr)];
   }
-  __syncthreads();
   if (cg == 0 && row < p.m_tokens) {
     const int64_t idx = (int64_t)bh * p.m_tokens + row;
     if (p.lse) p.lse[idx] = (m + log2f(l)) * 0.6931471805599453f;
     if (p.cached_mass) p.cached_mass[idx] = l_cac * inv;
-  }
   }
 }
 
@@ -1109,7 +1105,7 @@ int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk,
   attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mqr, mk, mv, p);
   KVQ_CUDA_TRY(cudaGetLastError());
   if (p.n_whole != p.n_units) {   // units were split over CTAs: combine their partial results
-    attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 4), 256, 0, st>>>(p, (int)grid.x);
+    attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 16), 256, 0, st>>>(p, (int)grid.x);
     KVQ_CUDA_TRY(cudaGetLastError());
   }
   return KVQ_OK;
