@@ -43,7 +43,7 @@ def load_peaks():
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel (profiles/)
 NCU_TRAFFIC_BYTES = {
-    "sweep_int2": 33.08e6,    # profiles/attn_tcgen05_sweep_int2.md, capture 3
+    "sweep_int2": 33.10e6,    # profiles/attn_tcgen05_sweep_int2.md, capture 4
     "dit": 209.3e6,           # profiles/attn_tcgen05_dit.md
 }
 
