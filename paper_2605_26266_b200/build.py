@@ -1,6 +1,9 @@
 """Builds libkvq.so in-tree with nvcc for sm_100a (no JIT cache, no torch extension)."""
 from __future__ import annotations
 
+import concurrent.futures
+import fcntl
+import hashlib
 import os
 import subprocess
 import sys
@@ -22,22 +25,48 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def _stale(target: str, deps: list[str]) -> bool:
-    if not os.path.exists(target):
-        return True
-    t = os.path.getmtime(target)
-    return any(os.path.getmtime(d) > t for d in deps)
+def _digest(paths: list[str], extra: str = "") -> str:
+    h = hashlib.sha256(extra.encode())
+    for p in paths:
+        with open(p, "rb") as f:
+            h.update(os.path.relpath(p, ROOT).encode() + b"\0" + f.read())
+    return h.hexdigest()
+
+
+def _current(target: str, digest: str) -> bool:
+    """True if `target` exists and was built from exactly these inputs (file times are not trusted: a copy of the
+    tree may have shuffled them)."""
+    try:
+        with open(target + ".stamp") as f:
+            return os.path.exists(target) and f.read().strip() == digest
+    except OSError:
+        return False
+
+
+def _stamp(target: str, digest: str) -> None:
+    with open(target + ".stamp", "w") as f:
+        f.write(digest + "\n")
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source and link libkvq.so next to this file; returns its path."""
-    objs = []
-    extra = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
-    for src in SOURCES:
+    """Compile every CUDA source and link libkvq.so next to this file; returns its path.  Several processes
+    (one per GPU) may call this at once: a file lock lets one of them build and the others find the result."""
+    with open(os.path.join(PKG, ".build.lock"), "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            return _build_locked(force, verbose)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
+
+
+def _build_locked(force: bool, verbose: bool) -> str:
+    headers = sorted(set(HEADERS + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]))
+
+    def compile_one(src: str):
         s = os.path.join(CSRC, src)
         o = os.path.join(CSRC, src[:-3] + ".o")
-        objs.append(o)
-        if force or _stale(o, [s] + HEADERS + extra):
+        d = _digest([s] + headers, " ".join(NVCC_FLAGS[:-4]))     # the flags without the include paths
+        if force or not _current(o, d):
             cmd = [_nvcc()] + NVCC_FLAGS + ["-c", s, "-o", o]
             r = subprocess.run(cmd, capture_output=True, text=True)
             log = r.stdout + r.stderr
@@ -47,12 +76,21 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
                 sys.stderr.write(log)
             if r.returncode != 0:
                 raise RuntimeError(f"nvcc failed for {src}")
-    if force or _stale(LIB, objs):
+            _stamp(o, d)
+        return o, d
+
+    with concurrent.futures.ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:     # nvcc runs as child processes
+        results = list(pool.map(compile_one, SOURCES))
+    objs = [o for o, _ in results]
+    digests = [d for _, d in results]
+    lib_digest = hashlib.sha256("".join(digests).encode()).hexdigest()
+    if force or not _current(LIB, lib_digest):
         cmd = [_nvcc(), "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")
+        _stamp(LIB, lib_digest)
     return LIB
 
 
