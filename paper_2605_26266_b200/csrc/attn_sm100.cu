@@ -1,7 +1,7 @@
 // Corrected chunk attention for sm_100a: TMA + tcgen05.mma with TMEM accumulators.
 //
-// A CTA works on 256 query rows of one (batch, head) at a time — two 128-row tiles that ping-pong on the
-// tensor pipe — and walks keys in tiles of 128: first the current chunk's BF16 keys and
+// A CTA works on 256 query rows of one (batch, head) at a time — two 128-row tiles that share the key and value
+// tiles — and walks keys in tiles of 128: first the current chunk's BF16 keys and
 // values (TMA straight into the 128-byte-swizzled operand layout, unrotated query, no bias),
 // then the cached keys and values, which four "dequant" warps expand from the packed
 // 2-/4-bit codes into the same operand layout in shared memory (never to HBM).  Between the
@@ -9,7 +9,7 @@
 // of Algorithm 1, both written by a small pre-pass kernel of the same call, replace the unrotated tile.
 //
 // Score of a cached key (Eq. (15) / Eq. (25)):  s = sigma*q~.k^ - (sigma^2/24) sum_j step_j^2 nu_j.
-// The bias is folded into the score contraction as one extra K=16 MMA step per tile:
+// The bias is folded into the score contraction as one extra K=16 MMA step per half tile:
 // A_extra[m, j] = -(sigma/24) nu_{m,j} (split into a BF16 high and low part, two columns) and
 // B_extra[i, j] = step_{i,j}^2 (exact in BF16), so the softmax warps spend no instruction on
 // it; correction off simply skips that step.
@@ -21,12 +21,20 @@
 // columns and consumed from there by the PV MMA.  Rotated queries are clamped to the FP16
 // range; dequantized keys must lie inside it.
 //
-// Roles (512 threads): warp 0 lane 0 issues TMA; warp 1 runs the MMA schedule converged and one elected
-// lane issues every tcgen05.mma; warps 4-11 are the softmax warps: warp 4+q and warp 8+q share TMEM lanes
-// 32q..32q+31 (one query row per lane) and take columns [0,64) and [64,128) of each score tile, exchanging
-// their partial row maxima through shared memory, for both query tiles in turn; warps 12-15 dequantize.
-// Registers are re-split between the roles with setmaxnreg.  The roles' loops are written to stay small:
-// the SM's instruction cache, and the GPC-level one behind it, bound this kernel before any pipe does.
+// Roles (512 threads): warp 0 lane 0 issues TMA; warps 1 and 2 issue the tcgen05.mma of query tile 0 and 1 (each
+// warp runs its schedule converged, one lane elected once issues); warps 4-7 are the softmax warps of query tile
+// 0, warps 8-11 those of query tile 1: warp w reads TMEM lanes 32 (w % 4) .. + 31, one query row per lane, so
+// row maxima and row sums need no exchange; warps 12-15 dequantize.  Registers are re-split between the roles
+// with setmaxnreg.
+//
+// A key tile of 128 keys is processed in two halves of 64 keys, each with its own 64 score columns in TMEM:
+// as soon as the softmax warps hand over P of one half (BF16 pairs written over the first 32 of that half's
+// columns), the issuer adds P V of those 64 keys to O and computes the same half's scores of the NEXT key tile
+// into the columns just freed, while the softmax warps work on the other half.  The scores a group needs next
+// are therefore usually ready when it asks for them.
+//
+// The roles' loops are written to stay small (rolled over halves, query tiles and MMA groups): the SM's
+// instruction cache, and the GPC-level one behind it, bound this kernel before any pipe does.
 //
 // Work is cut into units (batch*head, 256-row query block) of `tiles` key tiles each.  Persistent CTAs take
 // whole units in rounds; where that would leave SMs idle (a short last round, or fewer units than SMs) the
@@ -60,21 +68,21 @@ constexpr int kOffV = kOffK + 2 * kTileBytes;      // 2 stages
 constexpr int kOffAx = kOffV + 2 * kTileBytes;     // 2 query tiles
 constexpr int kOffBx = kOffAx + 2 * kXBytes;       // 2 stages
 constexpr int kOffBar = kOffBx + 2 * kXBytes;
-constexpr int kNumBars = 21;                       // mbarriers, 8 bytes each (enum Bar below)
+constexpr int kNumBars = 28;                       // mbarriers, 8 bytes each (enum Bar below)
 static_assert(kNumBars * 8 <= 256, "barrier area");
-constexpr int kOffXmax = kOffBar + 256;            // float [2 column halves][256 rows]: row-max exchange
-constexpr int kOffXl = kOffXmax + 2 * 256 * 4;     // float [2][256][2]: row-sum exchange (current, cached)
-constexpr int kOffMisc = kOffXl + 2 * 256 * 2 * 4;
+constexpr int kOffMisc = kOffBar + 256;
 constexpr int kSmemBytes = kOffMisc + 64 + 1024;   // + slack to align the base to 1024
 
-enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull = 9, kPFull = 11,
-           kODone = 13, kQCurDone = 15, kQRotFull = 16, kDrain = 17, kQEmpty = 18, kOFree = 19 };
+// kSFull, kPFull and kODone have four barriers each: index 2 * (half of the key tile) + (query tile); each of
+// them completes once per key tile, so that a waiter is never more than one phase behind
+enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull = 9, kPFull = 13,
+           kODone = 17, kQCurDone = 21, kQRotFull = 22, kDrain = 23, kQEmpty = 25, kOFree = 26 };
 
 constexpr uint32_t kTimeoutCycles = 2000000000u;   // about a second; 32-bit clock differences stay exact below 2^32
 constexpr uint32_t kDrainCycles = 20000000u;
 constexpr float kLog2e = 1.4426950408889634f;
-// registers per thread after reallocation: 128 * 72 + 256 * 168 + 128 * 96 = 64512 <= 65536
-constexpr int kRegsIssue = 72, kRegsSoftmax = 168, kRegsDequant = 96;
+// registers per thread after reallocation: 128 * 96 + 256 * 144 + 128 * 112 = 63488 <= 65536
+constexpr int kRegsIssue = 96, kRegsSoftmax = 144, kRegsDequant = 112;
 constexpr float kRescaleThreshold = 8.0f;          // lazy rescale of O: only when the max grows by > 2^8
 
 struct TParams {
@@ -165,12 +173,21 @@ struct Ctx {
   }
 };
 
-// The two softmax warps that share 32 query rows (warp 4 + q and warp 8 + q) meet at hardware barrier 1 + q to
-// exchange row maxima and row sums: about a third of the latency of an mbarrier round trip, once per query tile
-// and key tile.  Both warps run the same sequence of bounded waits before every meeting, so in a healthy run
-// neither can miss one; pair_release covers the aborting CTA (see the end of the softmax role).
-__device__ __forceinline__ void pair_sync(int q) { asm volatile("bar.sync %0, 64;" :: "r"(1 + q) : "memory"); }
-__device__ __forceinline__ void pair_release(int q) { asm volatile("bar.arrive %0, 64;" :: "r"(1 + q) : "memory"); }
+// Development aid, compiled in only with -DKVQ_TRACE: lane 0 of every warp of CTA 0 records (event id, clock)
+// pairs in a device array that kvq_debug_trace_read() copies to the host.  The library proper has none of it.
+#ifdef KVQ_TRACE
+constexpr int kTraceLen = 4096;
+__device__ uint32_t g_trace[16][kTraceLen];
+#define KVQ_TRACE_DECL int trace_n = 0
+#define KVQ_STAMP(id)                                                                            \
+  do {                                                                                           \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && trace_n < kTraceLen)                       \
+      g_trace[threadIdx.x >> 5][trace_n++] = ((uint32_t)(id) << 26) | ((uint32_t)clock() & 0x3FFFFFFu); \
+  } while (0)
+#else
+#define KVQ_TRACE_DECL
+#define KVQ_STAMP(id)
+#endif
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
@@ -359,6 +376,33 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
   }
 }
 
+// Softmax building blocks on one chunk of 32 score columns held in registers (the softmax role walks a row in
+// four such chunks through rolled loops: its code has to stay small, see the header).
+__device__ __forceinline__ void chunk_mask(uint32_t* a, int n_valid) {   // columns >= n_valid become -inf
+  if (n_valid < 32) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (i >= n_valid) a[i] = 0xFF800000u;
+  }
+}
+__device__ __forceinline__ void chunk_max(const uint32_t* a, float* mx) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 8) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mx[c] = max3(mx[c], __uint_as_float(a[i + 2 * c]), __uint_as_float(a[i + 2 * c + 1]));
+  }
+}
+// a[0..31] scores -> a[0..15] probabilities 2^(c s - m) as BF16 pairs; their sum is added to sum2
+__device__ __forceinline__ void chunk_exp(uint32_t* a, float2 c2, float2 nm2, float2& sum2) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    const float2 x = __ffma2_rn(make_float2(__uint_as_float(a[i]), __uint_as_float(a[i + 1])), c2, nm2);
+    const float2 pr = make_float2(ex2(x.x), ex2(x.y));
+    sum2 = __fadd2_rn(sum2, pr);
+    a[i >> 1] = cvt_bf16x2(pr.x, pr.y);
+  }
+}
+
 // Pre-pass over the query chunk (one launch before the attention kernel): q~ = (1/sqrt d) H (signs . q) in
 // FP32, stored as FP16 with the contraction dimension permuted the way the dequantized keys are laid out,
 // and -(sigma/24) nu_{m,j} (per-group squared norms of q~) as a BF16 high part plus a BF16 low part.  The
@@ -470,6 +514,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   Ctx cx{sbase + kOffBar, misc + 1};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  KVQ_TRACE_DECL;
   const int n_rt = (p.n_cur + kBlockN - 1) / kBlockN;
   const int n_ct = (p.n_cached + kBlockN - 1) / kBlockN;
   const int T = n_rt + n_ct;
@@ -481,18 +526,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     for (int s = 0; s < 2; ++s) {
       mbar_init(cx.bar(kKFull + s), 129);   // 128 dequant threads + the TMA thread, every tile
       mbar_init(cx.bar(kVFull + s), 129);
-      mbar_init(cx.bar(kKEmpty + s), 1);
-      mbar_init(cx.bar(kVEmpty + s), 1);
+      mbar_init(cx.bar(kKEmpty + s), 2);    // both MMA issuers commit
+      mbar_init(cx.bar(kVEmpty + s), 2);
       mbar_init(cx.bar(kSFull + s), 1);
-      mbar_init(cx.bar(kPFull + s), 256);
+      mbar_init(cx.bar(kSFull + 2 + s), 1);
+      mbar_init(cx.bar(kPFull + s), 128);   // the four softmax warps of a query tile
+      mbar_init(cx.bar(kPFull + 2 + s), 128);
       mbar_init(cx.bar(kODone + s), 1);
+      mbar_init(cx.bar(kODone + 2 + s), 1);
     }
-    mbar_init(cx.bar(kQCurDone), 1);
+    mbar_init(cx.bar(kQCurDone), 2);
     mbar_init(cx.bar(kQRotFull), 129);   // 128 dequant threads (bias rows) + the TMA thread (rotated query tile)
-    mbar_init(cx.bar(kDrain), 1);
-    mbar_init(cx.bar(kQEmpty), 1);
-    mbar_init(cx.bar(kOFree + 0), 256);
-    mbar_init(cx.bar(kOFree + 1), 256);
+    mbar_init(cx.bar(kDrain + 0), 1);
+    mbar_init(cx.bar(kDrain + 1), 1);
+    mbar_init(cx.bar(kQEmpty), 2);
+    mbar_init(cx.bar(kOFree + 0), 128);
+    mbar_init(cx.bar(kOFree + 1), 128);
     fence_barrier_init();
     prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_qr); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
   }
@@ -573,11 +622,20 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     }
-  } else if (warp == 1) {
-    // ================= MMA issuer =================
-    // The whole warp runs this code converged (operands stay warp-uniform); one elected lane issues.
+  } else if (warp <= 2) {
+    // ================= MMA issuers =================
+    // Warp 1 issues for query tile 0, warp 2 for query tile 1.  Each runs this code converged; one lane, elected
+    // once, issues every tcgen05.mma and commit of its query tile.
+    //
+    // A key tile is worked on in two halves of 64 keys, each with its own 64 score columns in TMEM, so that the
+    // scores of the next tile's half can be computed while the softmax warps are still busy with the other half
+    // of this tile: per (half, query tile) the issuer waits for that half of P, issues O += P V over its 64 keys
+    // and then at once S = Q K^T of the same half of the NEXT tile into the columns P has just left.  The tensor
+    // pipe executes this thread's MMAs in order, so the new scores cannot overtake the product that reads P.
     {
-      const uint32_t idesc_bf16 = make_idesc_bf16(128, 128, 0, 0);
+      const bool leader = elect_one();
+      const int qt = warp - 1;
+      const uint32_t idesc_bf16 = make_idesc_bf16(128, 64, 0, 0);
       const uint32_t idesc_f16 = idesc_bf16 & ~((7u << 7) | (7u << 10));     // A, B format 0 = FP16
       const uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);              // B (values) is MN-major
       // Descriptors are built once; stepping along K only adds a constant to the 14-bit address field
@@ -587,12 +645,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint64_t dv0 = make_smem_desc(sbase + kOffV, kHalfTile, 1024, kLayoutSw128);
       const uint64_t dax0 = make_smem_desc(sbase + kOffAx, 128, 256, kLayoutNone);
       const uint64_t dbx0 = make_smem_desc(sbase + kOffBx, 128, 256, kLayoutNone);
-      auto commit1 = [&](uint32_t bar) { if (elect_one()) tc_commit(bar); __syncwarp(); };
-      auto issue_qk = [&](int qt, int s, bool cached) {
-        if (elect_one()) {
+      // S[:, 64 hf .. 64 hf + 63] = Q_qt K^T over keys 64 hf .. 64 hf + 63 of stage s (+ the bias step)
+      auto issue_qk = [&](int s, int hf, bool cached) {
+        if (!leader) return;
         const uint32_t idesc = cached ? idesc_f16 : idesc_bf16;
-        const uint64_t qd = dq0 + (uint64_t)(qt * (kTileBytes >> 4)), kd = dk0 + (uint64_t)(s * (kTileBytes >> 4));
-        const uint32_t d_tmem = tmem + qt * 128;
+        const uint64_t qd = dq0 + (uint64_t)(qt * (kTileBytes >> 4));
+        const uint64_t kd = dk0 + (uint64_t)(s * (kTileBytes >> 4) + hf * (64 * 128 >> 4));   // key rows are 128 bytes
+        const uint32_t d_tmem = tmem + qt * 128 + hf * 64;
         constexpr int kBlk = kHalfTile >> 4;
         mma_ss_off<0>(d_tmem, qd, kd, idesc, 0);
         mma_ss_off<2>(d_tmem, qd, kd, idesc, 1);
@@ -602,28 +661,21 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mma_ss_off<kBlk + 2>(d_tmem, qd, kd, idesc, 1);
         mma_ss_off<kBlk + 4>(d_tmem, qd, kd, idesc, 1);
         mma_ss_off<kBlk + 6>(d_tmem, qd, kd, idesc, 1);
-        if (cached && p.correction)
-          mma_ss(d_tmem, dax0 + (uint64_t)(qt * (kXBytes >> 4)), dbx0 + (uint64_t)(s * (kXBytes >> 4)), idesc_bf16, 1);
-        tc_commit(cx.bar(kSFull + qt));
-        }
-        __syncwarp();
+        if (cached && p.correction)   // rows 64 hf .. of the 128 x 16 bias tile: 8-row groups are 256 bytes apart
+          mma_ss(d_tmem, dax0 + (uint64_t)(qt * (kXBytes >> 4)), dbx0 + (uint64_t)(s * (kXBytes >> 4) + hf * (8 * 256 >> 4)), idesc_bf16, 1);
+        tc_commit(cx.bar(kSFull + 2 * hf + qt));
       };
-      auto issue_pv = [&](int qt, int s, bool accumulate) {
-        if (elect_one()) {
-        const uint64_t vd = dv0 + (uint64_t)(s * (kTileBytes >> 4));
-        const uint32_t d_tmem = tmem + 256 + qt * 128, a_tmem = tmem + qt * 128;
-        const uint32_t acc = accumulate ? 1u : 0u;
-        mma_ts_off<0 * 128>(d_tmem, a_tmem + 0, vd, idesc_pv, acc);
+      // O_qt += P V over keys 64 hf .. 64 hf + 63 of stage s; P (BF16 pairs) sits in the first 32 of that half's
+      // score columns
+      auto issue_pv = [&](int s, int hf, bool accumulate) {
+        if (!leader) return;
+        const uint64_t vd = dv0 + (uint64_t)(s * (kTileBytes >> 4) + hf * (4 * 128));
+        const uint32_t d_tmem = tmem + 256 + qt * 128, a_tmem = tmem + qt * 128 + hf * 64;
+        mma_ts_off<0 * 128>(d_tmem, a_tmem + 0, vd, idesc_pv, accumulate ? 1u : 0u);
         mma_ts_off<1 * 128>(d_tmem, a_tmem + 8, vd, idesc_pv, 1);
         mma_ts_off<2 * 128>(d_tmem, a_tmem + 16, vd, idesc_pv, 1);
         mma_ts_off<3 * 128>(d_tmem, a_tmem + 24, vd, idesc_pv, 1);
-        mma_ts_off<4 * 128>(d_tmem, a_tmem + 32, vd, idesc_pv, 1);
-        mma_ts_off<5 * 128>(d_tmem, a_tmem + 40, vd, idesc_pv, 1);
-        mma_ts_off<6 * 128>(d_tmem, a_tmem + 48, vd, idesc_pv, 1);
-        mma_ts_off<7 * 128>(d_tmem, a_tmem + 56, vd, idesc_pv, 1);
-        tc_commit(cx.bar(kODone + qt));
-        }
-        __syncwarp();
+        tc_commit(cx.bar(kODone + 2 * hf + qt));
       };
       Schedule sch(blockIdx.x, gridDim.x, p);
       Segment sg;
@@ -635,49 +687,50 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // score MMAs nothing reads the unrotated query any more
         const int t_lastcur = (sg.tb < n_rt) ? min(sg.te, n_rt) - 1 : -1;
         const int t_rot = max(sg.tb, n_rt);          // first cached tile: its scores need the rotated query
-        if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, sp, 201)))) break;
-        // Iteration t issues O += P V of tile t and S = Q K^T of tile t + 1 (t = tb - 1: only the scores of
-        // the first tile).  The four MMA groups of an iteration go through ONE rolled loop, so that the
-        // issue code exists once and the warp's loop stays small in the instruction cache.  Order:
-        // PV0 QK0 PV1 QK1; if tile t + 1 is the first cached one, PV0 PV1 QK0 QK1, because its scores have
-        // to wait for the query rotation, which itself waits for every earlier score MMA.
+        if (!(ok = cx.wait(kQFull, sp, 201))) break;
+        // Iteration t issues the products of tile t and the scores of tile t + 1 (t = tb - 1: only the scores of
+        // the first tile), in the order (half 0, tile 0) (half 0, tile 1) (half 1, tile 0) (half 1, tile 1), each
+        // as "P V, then Q K^T".  If tile t + 1 is the first cached one, all four products come first: its scores
+        // wait for the rotated query, which itself waits for every earlier score MMA.
         --it;
         for (int t = sg.tb - 1; ok && t < sg.te; ++t, ++it) {
-          const bool has_pv = t >= sg.tb, has_qk = t + 1 < sg.te;
-          const bool first = t == sg.tb;
-          const bool rot = has_qk && (t + 1 == t_rot);
-          const bool next_cached = t + 1 >= n_rt;
           const int s = it & 1, s1 = (it + 1) & 1;
           const uint32_t ph = (it >> 1) & 1, ph1 = ((it + 1) >> 1) & 1;
-          if (rot && !has_pv) commit1(cx.bar(kQCurDone));        // the segment starts in the cache
+          const bool has_pv = t >= sg.tb, has_qk = t + 1 < sg.te, first = t == sg.tb;
+          const bool rot = has_qk && t + 1 == t_rot;
+          KVQ_STAMP(32);
+          if (rot && !has_pv && leader) tc_commit(cx.bar(kQCurDone));      // the segment starts in the cache
           // last iteration: every score MMA of the segment is issued, so the query buffer (and the bias rows) can
           // be handed to the next segment while the last P V products still run
-          if (!has_qk) commit1(cx.bar(kQEmpty));
+          if (!has_qk && leader) tc_commit(cx.bar(kQEmpty));
+          const int n_ops = rot ? 4 : 2;
 #pragma unroll 1
-          for (int step = 0; step < 4; ++step) {
-            const int op = rot ? step : (((step & 1) << 1) | (step >> 1));   // bit 1: scores, bit 0: query tile
-            const int qt = op & 1;
-            if (op < 2) {
-              if (!has_pv) continue;
-              if (qt == 0 && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kVFull + s, ph, 203)))) break;
-              if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kPFull + qt, it & 1, 204)))) break;
-              // first tile of a segment: the previous segment's O must have been read out
-              if (first && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kOFree + qt, sp ^ 1, 209)))) break;
+          for (int op = 0; op < n_ops; ++op) {
+            const int hf = op & 1;
+            if (has_pv && op < 2) {
+              if (op == 0 && !(ok = cx.wait(kVFull + s, ph, 203))) break;
+              if (!(ok = cx.wait(kPFull + 2 * hf + qt, it & 1, 204))) break;
+              // first product of a segment: the previous segment's O must have been read out
+              if (first && hf == 0 && !(ok = cx.wait(kOFree + qt, sp ^ 1, 209))) break;
+              KVQ_STAMP(34);
               tc_fence_after();
-              issue_pv(qt, s, !first);
-              if (qt == 1) commit1(cx.bar(kVEmpty + s));
-            } else {
-              if (!has_qk) continue;
-              if (qt == 0) {
-                if (rot && !(ok = __all_sync(0xFFFFFFFFu, cx.wait(kQRotFull, sp, 207)))) break;
-                if (!(ok = __all_sync(0xFFFFFFFFu, cx.wait(kKFull + s1, ph1, 205)))) break;
+              issue_pv(s, hf, !(first && hf == 0));
+              if (op == 1 && leader) tc_commit(cx.bar(kVEmpty + s));
+              KVQ_STAMP(10 + qt);
+            }
+            if (has_qk && (!rot || op >= 2)) {
+              if (hf == 0) {
+                if (rot && !(ok = cx.wait(kQRotFull, sp, 207))) break;
+                if (!(ok = cx.wait(kKFull + s1, ph1, 205))) break;
                 tc_fence_after();
               }
-              issue_qk(qt, s1, next_cached);
-              if (qt == 1) {
-                commit1(cx.bar(kKEmpty + s1));
-                if (t + 1 == t_lastcur) commit1(cx.bar(kQCurDone));
+              KVQ_STAMP(36);
+              issue_qk(s1, hf, t + 1 >= n_rt);
+              if (hf == 1 && leader) {
+                tc_commit(cx.bar(kKEmpty + s1));
+                if (t + 1 == t_lastcur) tc_commit(cx.bar(kQCurDone));
               }
+              KVQ_STAMP(14 + qt);
             }
           }
         }
@@ -685,52 +738,52 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         ++nseg;
       }
       // everything issued so far must have retired before TMEM is freed
-      commit1(cx.bar(kDrain));
-      cx.drain(kDrain, 0);
+      if (leader) tc_commit(cx.bar(kDrain + qt));
+      cx.drain(kDrain + qt, 0);
     }
   }
   } else if (warp < 12) {
     // ================= softmax groups =================
-    // Both groups work on every query tile: warp 4+q and warp 8+q share TMEM lanes 32q..32q+31 (one row per
-    // lane) and take columns [0,64) and [64,128) of that row's scores.  The two warps exchange their partial
-    // row maxima through shared memory (pair barrier), so a tile's softmax latency is that of 64 elements.
+    // Warps 4-7 own query tile 0, warps 8-11 query tile 1; warp w reads TMEM lanes 32 (w % 4) .. + 31, one query
+    // row per lane, so the row maximum and the row sums need no exchange between threads.  A key tile is taken
+    // in two halves of 64 keys, each one step of the online softmax: 64 scores into registers, maximum,
+    // exponentials, 32 columns of BF16 pairs back over the scores.  While a group works on one half the tensor
+    // pipe computes the other half's next scores, so a group seldom waits.
     setmaxnreg_inc<kRegsSoftmax>();
-    const int half = (warp - 4) >> 2;                         // which 64 columns
+    const int qt = (warp - 4) >> 2;                           // which query tile
     const int wq = warp & 3;                                  // which 32 rows (TMEM lane quarter)
-    const int r128 = wq * 32 + lane;
+    const int r256 = qt * kBlockM + wq * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+    const uint32_t s_addr = tmem + lane_addr + qt * 128;      // scores of half hf at columns 64 hf; P over their first 32
+    const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128;
     const float c_row = p.scale_log2;
-    float* xmax = reinterpret_cast<float*>(smem + kOffXmax);
-    float* xl = reinterpret_cast<float*>(smem + kOffXl);
     Schedule sch(blockIdx.x, gridDim.x, p);
     Segment sg;
     int it = 0, nseg = 0;
     bool ok = true;
     while (ok && sch.next(sg)) {
-      // Running max and row sums (current / cached keys) of the query tile being worked on (m_a ...) and of
-      // the other one (m_b ...).  The loops over the two query tiles are rolled, to keep this role's code
-      // small in the instruction cache, and swap the two sets at the end of each pass.
-      float m_a = -INFINITY, m_b = -INFINITY, lcur_a = 0.f, lcur_b = 0.f, lcac_a = 0.f, lcac_b = 0.f;
-      uint32_t sr[64];                           // this thread's 64 scores, then its 32 packed probabilities
+      float m_run = -INFINITY, lcur = 0.f, lcac = 0.f;   // running max (log2 units), row sums over current / cached keys
+      bool fresh = true;                                 // no product has been added to O in this segment yet
       for (int t = sg.tb; ok && t < sg.te; ++t, ++it) {
         const bool cached = t >= n_rt;
-        const int n_valid = (cached ? min(kBlockN, p.n_cached - (t - n_rt) * kBlockN) : min(kBlockN, p.n_cur - t * kBlockN)) - half * 64;
+        const int n_valid = cached ? min(kBlockN, p.n_cached - (t - n_rt) * kBlockN) : min(kBlockN, p.n_cur - t * kBlockN);
 #pragma unroll 1
-        for (int qt = 0; qt < 2; ++qt) {
-          const int r256 = qt * kBlockM + r128;
-          const uint32_t s_addr = tmem + lane_addr + qt * 128 + half * 64;
-          const uint32_t p_addr = tmem + lane_addr + qt * 128 + half * 32;
-          const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128 + half * 64;
-          ok = __all_sync(0xFFFFFFFFu, cx.wait(kSFull + qt, it & 1, 301));
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t sr[64];                         // this thread's 64 scores, then its 32 packed probabilities
+          KVQ_STAMP(0);
+          ok = __all_sync(0xFFFFFFFFu, cx.wait(kSFull + 2 * hf + qt, it & 1, 301));
           if (!ok) break;
+          KVQ_STAMP(1);
           tc_fence_after();
-          tmem_ld32(s_addr, sr);
-          tmem_ld32(s_addr + 32, sr + 32);
+          tmem_ld32(s_addr + 64 * hf, sr);
+          tmem_ld32(s_addr + 64 * hf + 32, sr + 32);
           tmem_wait_ld();
-          if (n_valid < 64) {                      // ragged last tile of the current chunk or of the cache
+          KVQ_STAMP(2);
+          const int nv = n_valid - 64 * hf;
+          if (nv < 64) {                           // ragged last tile of the current chunk or of the cache
 #pragma unroll
             for (int i = 0; i < 64; ++i)
-              if (i >= n_valid) sr[i] = 0xFF800000u;  // -inf
+              if (i >= nv) sr[i] = 0xFF800000u;    // -inf
           }
           float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -738,20 +791,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
             for (int c = 0; c < 4; ++c) mx[c] = max3(mx[c], __uint_as_float(sr[i + 2 * c]), __uint_as_float(sr[i + 2 * c + 1]));
           }
-          const float mine = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-          xmax[half * 256 + r256] = mine;
-          tc_fence_before();
-          pair_sync(wq);
-          tc_fence_after();
-          const float m_new = fmaxf(m_a, fmaxf(mine, xmax[(half ^ 1) * 256 + r256]) * c_row);
-          if (__any_sync(0xFFFFFFFFu, m_new - m_a > kRescaleThreshold)) {
-            if (t > sg.tb) {
-              ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (it - 1) & 1, 302));
+          const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c_row);
+          if (__any_sync(0xFFFFFFFFu, m_new - m_run > kRescaleThreshold)) {
+            if (!fresh) {
+              // the product of the previous half (the last one issued on this O) must have retired
+              ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + 2 * (hf ^ 1) + qt, (it - (hf ^ 1)) & 1, 302));
               if (!ok) break;
               tc_fence_after();
-              const float f = ex2(m_a - m_new);
+              const float f = ex2(m_run - m_new);
 #pragma unroll 1
-              for (int c = 0; c < 4; ++c) {
+              for (int c = 0; c < 8; ++c) {
                 uint32_t r[16];
                 tmem_ld16(o_addr + 16 * c, r);
                 tmem_wait_ld();
@@ -759,12 +808,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
                 tmem_st16(o_addr + 16 * c, r);
               }
-              lcur_a *= f; lcac_a *= f;
+              lcur *= f; lcac *= f;
             }
-            m_a = m_new;
+            m_run = m_new;
           }
-          const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m_a, -m_a);
+          const float2 c2 = make_float2(c_row, c_row), nm2 = make_float2(-m_run, -m_run);
           float2 sum2 = make_float2(0.f, 0.f);
+          KVQ_STAMP(3);
 #pragma unroll
           for (int i = 0; i < 64; i += 2) {
             const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), c2, nm2);
@@ -772,46 +822,44 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             sum2 = __fadd2_rn(sum2, pr);
             sr[i >> 1] = cvt_bf16x2(pr.x, pr.y);
           }
-          tmem_st32(p_addr, sr);
-          if (cached) lcac_a += sum2.x + sum2.y; else lcur_a += sum2.x + sum2.y;
+          tmem_st32(s_addr + 64 * hf, sr);
+          if (cached) lcac += sum2.x + sum2.y; else lcur += sum2.x + sum2.y;
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(cx.bar(kPFull + qt));
-          { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
+          mbar_arrive(cx.bar(kPFull + 2 * hf + qt));
+          KVQ_STAMP(4 + hf);
+          fresh = false;
         }
       }
       if (!ok) break;
-      // ---- segment epilogue: read O out of TMEM, release it, combine the two column halves' row sums ----
+      // ---- segment epilogue: read this row of O out of TMEM, release it, write the normalised row ----
       const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
       const bool whole = sg.tb == 0 && sg.te == T;
       uint8_t* slot = p.partial + (size_t)(2 * blockIdx.x + sg.slot) * kSlotBytes;   // partial segments only
+      ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + 2 + qt, (it - 1) & 1, 303));            // the last product of the segment is a second half
+      if (!ok) break;
+      tc_fence_after();
+      const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
+      // a whole unit writes its rows of the output; a partial segment writes the same normalised rows into its
+      // slot, with the statistics the merge kernel weighs them by
+      const float l = lcur + lcac;
+      const float inv = 1.0f / l;
+      const bool store = !whole || row < p.m_tokens;
+      // consecutive 8-column pieces: 16 bytes apart in a row of the output, 4096 bytes apart in a slot
+      uint8_t* dst = whole ? reinterpret_cast<uint8_t*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st)
+                           : slot + r256 * 16;
+      const int piece = whole ? 16 : 4096;
 #pragma unroll 1
-      for (int qt = 0; qt < 2; ++qt) {
-        const int r256 = qt * kBlockM + r128;
-        const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128 + half * 64;
-        ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + qt, (it - 1) & 1, 303));
-        if (!ok) break;
-        tc_fence_after();
-        tmem_ld32(o_addr, sr);
-        tmem_ld32(o_addr + 32, sr + 32);
+      for (int hf = 0; hf < 2; ++hf) {               // 64 columns at a time
+        uint32_t sr[64];
+        tmem_ld32(o_addr + 64 * hf, sr);
+        tmem_ld32(o_addr + 64 * hf + 32, sr + 32);
         tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(cx.bar(kOFree + qt));
-        xl[(half * 256 + r256) * 2] = lcur_a;
-        xl[(half * 256 + r256) * 2 + 1] = lcac_a;
-        pair_sync(wq);
-        const float lc = lcur_a + xl[((half ^ 1) * 256 + r256) * 2];
-        const float la = lcac_a + xl[((half ^ 1) * 256 + r256) * 2 + 1];
-        const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
-        // a whole unit writes its rows of the output; a partial segment writes the same normalised rows into its
-        // slot, with the statistics the merge kernel weighs them by
-        const float l = lc + la;
-        const float inv = 1.0f / l;
-        if (!whole || row < p.m_tokens) {
-          // consecutive 8-column pieces: 16 bytes apart in a row of the output, 4096 bytes apart in a slot
-          uint8_t* dst = whole ? reinterpret_cast<uint8_t*>(p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)row * p.o_st + half * 64)
-                               : slot + ((half * 8) * 256 + r256) * 16;
-          const int piece = whole ? 16 : 4096;
+        if (hf == 1) {                               // the whole row is in registers: O can be overwritten
+          tc_fence_before();
+          mbar_arrive(cx.bar(kOFree + qt));
+        }
+        if (store) {
 #pragma unroll
           for (int i = 0; i < 64; i += 8) {
             uint4 v;
@@ -819,26 +867,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             v.y = cvt_bf16x2(__uint_as_float(sr[i + 2]) * inv, __uint_as_float(sr[i + 3]) * inv);
             v.z = cvt_bf16x2(__uint_as_float(sr[i + 4]) * inv, __uint_as_float(sr[i + 5]) * inv);
             v.w = cvt_bf16x2(__uint_as_float(sr[i + 6]) * inv, __uint_as_float(sr[i + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + (i >> 3) * piece) = v;
-          }
-          if (half == 0) {
-            if (whole) {
-              const int64_t idx = (int64_t)bh * p.m_tokens + row;
-              if (p.lse) p.lse[idx] = (m_a + log2f(l)) * 0.6931471805599453f;
-              if (p.cached_mass) p.cached_mass[idx] = la * inv;
-            } else {
-              float* st = reinterpret_cast<float*>(slot + kSlotStats);
-              st[r256] = m_a; st[256 + r256] = lc; st[512 + r256] = la;
-            }
+            *reinterpret_cast<uint4*>(dst + (8 * hf + (i >> 3)) * piece) = v;
           }
         }
-        { float x_ = m_a; m_a = m_b; m_b = x_; x_ = lcur_a; lcur_a = lcur_b; lcur_b = x_; x_ = lcac_a; lcac_a = lcac_b; lcac_b = x_; }
+      }
+      if (store) {
+        if (whole) {
+          const int64_t idx = (int64_t)bh * p.m_tokens + row;
+          if (p.lse) p.lse[idx] = (m_run + log2f(l)) * 0.6931471805599453f;
+          if (p.cached_mass) p.cached_mass[idx] = lcac * inv;
+        } else {
+          float* st = reinterpret_cast<float*>(slot + kSlotStats);
+          st[r256] = m_run; st[256 + r256] = lcur; st[512 + r256] = lcac;
+        }
       }
       ++nseg;
     }
-    // Leaving because the CTA is aborting: the partner warp may be sitting in pair_sync, which has no time-out
-    // of its own.  One arrival on the pair's barrier lets it through; it then fails its next bounded wait.
-    if (*cx.abort) pair_release(wq);
     tc_fence_before();
   } else {
     // ================= dequant warps =================
@@ -871,6 +915,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int k1 = (ct + 1) * kBlockN + dt;    // this thread's key in the next tile
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kKEmpty + s, ph ^ 1, 401));
         if (!ok) break;
+        KVQ_STAMP(22);
         if (ct >= 0) {
           dequant_keys<BITS, GROUP>(rk, smem + kOffK + s * kTileBytes, dt);
           if (p.correction) {   // B_extra row: step_j^2, exact in BF16
@@ -883,6 +928,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (t + 1 < sg.te) load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k1), k1 < p.n_cached);
         }
         mbar_arrive(cx.bar(kKFull + s));
+        KVQ_STAMP(20);
         if (t == t_rot) {
           // ---- A_extra: -(sigma/24) nu rows of this unit's 256 queries, written by the pre-pass ----
           // (the new query tile being in means every MMA of the previous segment, which read the old rows, retired)
@@ -901,12 +947,14 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kVEmpty + s, ph ^ 1, 404));
         if (!ok) break;
+        KVQ_STAMP(23);
         if (ct >= 0) {
           dequant_values<BITS, GROUP>(rv, smem + kOffV + s * kTileBytes, dt);
           fence_proxy_async_smem();
           if (t + 1 < sg.te) load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(k1), k1 < p.n_cached);
         }
         mbar_arrive(cx.bar(kVFull + s));
+        KVQ_STAMP(21);
       }
       if (!ok) break;
       if (sg.te <= n_rt) mbar_arrive(cx.bar(kQRotFull));   // no rotation in this segment: keep the phase count in step
@@ -1275,3 +1323,13 @@ int launch_attn_tcgen05_static(const AttnArgs& a) {
 }
 
 }  // namespace kvq
+
+#ifdef KVQ_TRACE
+extern "C" int kvq_debug_trace_read(uint32_t* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, kvq::g_trace, sizeof(kvq::g_trace));
+}
+extern "C" int kvq_debug_trace_clear() {
+  static uint32_t zeros[16 * kvq::kTraceLen];
+  return (int)cudaMemcpyToSymbol(kvq::g_trace, zeros, sizeof(zeros));
+}
+#endif
