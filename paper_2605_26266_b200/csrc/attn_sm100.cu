@@ -376,33 +376,6 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
   }
 }
 
-// Softmax building blocks on one chunk of 32 score columns held in registers (the softmax role walks a row in
-// four such chunks through rolled loops: its code has to stay small, see the header).
-__device__ __forceinline__ void chunk_mask(uint32_t* a, int n_valid) {   // columns >= n_valid become -inf
-  if (n_valid < 32) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (i >= n_valid) a[i] = 0xFF800000u;
-  }
-}
-__device__ __forceinline__ void chunk_max(const uint32_t* a, float* mx) {
-#pragma unroll
-  for (int i = 0; i < 32; i += 8) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) mx[c] = max3(mx[c], __uint_as_float(a[i + 2 * c]), __uint_as_float(a[i + 2 * c + 1]));
-  }
-}
-// a[0..31] scores -> a[0..15] probabilities 2^(c s - m) as BF16 pairs; their sum is added to sum2
-__device__ __forceinline__ void chunk_exp(uint32_t* a, float2 c2, float2 nm2, float2& sum2) {
-#pragma unroll
-  for (int i = 0; i < 32; i += 2) {
-    const float2 x = __ffma2_rn(make_float2(__uint_as_float(a[i]), __uint_as_float(a[i + 1])), c2, nm2);
-    const float2 pr = make_float2(ex2(x.x), ex2(x.y));
-    sum2 = __fadd2_rn(sum2, pr);
-    a[i >> 1] = cvt_bf16x2(pr.x, pr.y);
-  }
-}
-
 // Pre-pass over the query chunk (one launch before the attention kernel): q~ = (1/sqrt d) H (signs . q) in
 // FP32, stored as FP16 with the contraction dimension permuted the way the dequantized keys are laid out,
 // and -(sigma/24) nu_{m,j} (per-group squared norms of q~) as a BF16 high part plus a BF16 low part.  The

@@ -115,12 +115,14 @@ def _head_aux(w: Workload):
     return idx, uq, uk
 
 
-def make_chunk(w: Workload, chunk_index: int, tokens: int | None = None):
-    """Q, K, V of chunk `chunk_index` as BF16 bit patterns, each [batch, heads, tokens, head_dim]."""
+def make_chunk(w: Workload, chunk_index: int, tokens: int | None = None, need_q: bool = True):
+    """Q, K, V of chunk `chunk_index` as BF16 bit patterns, each [batch, heads, tokens, head_dim].
+    need_q=False skips the query draw (Q comes back as None): every tensor has its own generator, so K and V
+    are the same bits either way.  Cached chunks only ever contribute K and V."""
     n = w.chunk if tokens is None else tokens
     shape = (w.batch, w.heads, n, w.head_dim)
     idx, uq, uk = _head_aux(w)
-    q = _rng(w, T_Q, chunk_index).standard_normal(shape, dtype=np.float32)
+    q = _rng(w, T_Q, chunk_index).standard_normal(shape, dtype=np.float32) if need_q else None
     if w.k_dist == "student_t3":
         k = _rng(w, T_K, chunk_index).standard_t(3.0, size=shape).astype(np.float32)
     else:
@@ -130,9 +132,10 @@ def make_chunk(w: Workload, chunk_index: int, tokens: int | None = None):
         for h in range(w.heads):
             k[:, h, :, idx[h, :w.k_outliers]] *= np.float32(w.k_outlier_scale)
     if w.head_scale:
-        q *= uq[None, :, None, None]
+        if need_q:
+            q *= uq[None, :, None, None]
         k *= uk[None, :, None, None]
-    return f32_to_bf16_bits(q), f32_to_bf16_bits(k), f32_to_bf16_bits(v)
+    return (f32_to_bf16_bits(q) if need_q else None), f32_to_bf16_bits(k), f32_to_bf16_bits(v)
 
 
 def sample_rows(m: int, tile: int = 128, n_random: int = 64, seed: int = 0) -> np.ndarray:
