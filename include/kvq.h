@@ -51,7 +51,8 @@ extern "C" {
 #define KVQ_ERR_ALIGNMENT     -3   /* pointer not 16-byte aligned, stride not a multiple of 8 elements */
 #define KVQ_ERR_CAPACITY      -4   /* the append or the window would run past `capacity` */
 #define KVQ_ERR_CUDA          -5   /* a CUDA runtime/driver call failed; see kvq_last_cuda_error() */
-#define KVQ_ERR_TIMEOUT       -6   /* a bounded device-side wait expired (reported through status_word) */
+#define KVQ_ERR_TIMEOUT       -6   /* a bounded device-side wait expired: what kvq_status_word_result() returns for a
+                                      non-zero status_word */
 #define KVQ_ERR_WORKSPACE     -7   /* workspace missing or smaller than kvq_attn_workspace_bytes() */
 
 /* kvq_cache_desc.flags */
@@ -239,6 +240,31 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
  */
 int kvq_unpack_codes(const kvq_cache_desc* desc, int which, int64_t begin, int64_t n,
                      uint8_t* out_codes, kvq_stream_t stream);
+
+/*
+ * Bounded device-side waits.  (The paper has no counterpart: this is how the tcgen05 kernel fails.)
+ *
+ * Inside the tcgen05 kernel the roles of a CTA (TMA producer, MMA issuer, softmax warps, dequantization warps)
+ * hand tiles to one another through shared-memory barriers.  No wait on such a barrier is unbounded: a wait
+ * that does not complete within its cycle budget (about one second by default) records a site code in the
+ * CTA, every role of that CTA leaves its loop at its next wait, work in flight is drained, and the kernel
+ * returns.  The first site code reaches the caller's status_word; the outputs are then undefined.
+ * Site codes: TMA producer 100 (query buffer free), 101 (key stage free), 102 (value stage free), 103 (last
+ * unrotated score product done); MMA issuer 201 (query tile), 203 (value tile), 204 (probabilities), 205 (key
+ * tile), 207 (rotated query), 209 (output accumulator read out); softmax warps 301 (scores), 302 (product
+ * retired before a rescale), 303 (last product before the epilogue); dequantization warps 401 (key stage free),
+ * 402 (query tile, for the bias rows), 404 (value stage free).
+ *
+ * kvq_status_word_result maps a status word read back by the caller (host value) to KVQ_OK (0) or
+ * KVQ_ERR_TIMEOUT (anything else).
+ * kvq_set_wait_budget_cycles sets the budget, in SM clock cycles, for kernels launched afterwards by this
+ * process (0 restores the default; values above 0xFFFF0000 are KVQ_ERR_INVALID_ARG).  It exists so that the
+ * time-out path can be exercised on purpose: with a budget of a few cycles the first wait that is not complete
+ * at its first poll gives up, and the call returns with a status word set, on a healthy GPU and without any
+ * wait left hanging.  Not meant for production use.
+ */
+int kvq_status_word_result(int32_t status_word_value);
+int kvq_set_wait_budget_cycles(uint64_t cycles);
 
 /* Host-side helpers. */
 const char* kvq_status_string(int status);   /* static string, never NULL */

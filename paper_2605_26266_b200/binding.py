@@ -76,6 +76,10 @@ def _load():
         C.c_void_p, kvq_strides, C.c_void_p, C.c_void_p, kvq_strides,
         C.c_int64, C.c_int64, C.c_void_p, kvq_strides,
         C.c_float, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.kvq_status_word_result.restype = C.c_int
+    lib.kvq_status_word_result.argtypes = [C.c_int32]
+    lib.kvq_set_wait_budget_cycles.restype = C.c_int
+    lib.kvq_set_wait_budget_cycles.argtypes = [C.c_uint64]
     lib.kvq_unpack_codes.restype = C.c_int
     lib.kvq_unpack_codes.argtypes = [C.POINTER(kvq_cache_desc), C.c_int, C.c_int64, C.c_int64,
                                      C.c_void_p, C.c_void_p]
@@ -228,6 +232,14 @@ def kvq_attn_corrected_static_scratch(cache: Cache, q, k_cur, v_cur, softmax_sca
         _strides(k_cur), q.shape[2], k_cur.shape[2], out.data_ptr(), _strides(out), float(softmax_scale), flags,
         _ptr(lse), _ptr(cached_mass), _ptr(status_word), _stream()), "kvq_attn_corrected_static_scratch")
     return out
+
+
+def kvq_status_word_result(word: int) -> int:
+    return lib.kvq_status_word_result(int(word))
+
+
+def kvq_set_wait_budget_cycles(cycles: int) -> None:
+    _check(lib.kvq_set_wait_budget_cycles(int(cycles)), "kvq_set_wait_budget_cycles")
 
 
 def kvq_unpack_codes(cache: Cache, which: int, begin: int, n: int) -> torch.Tensor:

@@ -467,11 +467,13 @@ int launch(const AParams& p, dim3 grid, cudaStream_t st) {
                           (size_t)(4 * D + 2 * kBM) * sizeof(float);
   // the exact correction adds its table: 64 rows x groups x 128 step values
   const size_t smem = base + (p.correction == 2 ? (size_t)kBM * (D / p.group) * 128 * sizeof(float) : 0);
-  static bool configured = false;
-  if (!configured) {
+  static PerDevice configured;                       // the attribute is per device
+  int dev = 0;
+  { const int r = current_device(&dev); if (r != KVQ_OK) return r; }
+  if (configured.first(dev)) {
     KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_mma_sync_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)(base + (size_t)kBM * 4 * 128 * sizeof(float))));
-    configured = true;
+    configured.done(dev);
   }
   attn_mma_sync_kernel<D, BITS><<<grid, kThreads, smem, st>>>(p);
   KVQ_CUDA_TRY(cudaGetLastError());

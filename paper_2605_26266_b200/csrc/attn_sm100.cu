@@ -97,6 +97,7 @@ struct TParams {
   float ax_coef;           // -sigma / 24
   float* lse; float* cached_mass;
   int32_t* status;
+  uint32_t wait_budget;    // cycles a device-side wait may take (kTimeoutCycles unless a test has shortened it)
   // schedule: units = (batch*head, 256-row query block); every unit has `tiles` key tiles (see Schedule)
   int q_blocks, n_units, tiles;
   int n_whole;             // units [0, n_whole) are computed whole; the rest are split over all CTAs
@@ -152,6 +153,7 @@ struct Schedule {
 struct Ctx {
   uint32_t bar0;
   volatile int* abort;     // shared-memory word: 0, or the diagnostic code of the wait that gave up
+  uint32_t budget;         // cycles a wait may take before it gives up
   __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * i; }
   // Bounded wait; false once the CTA is aborting.  Written to be small: it is inlined at some forty
   // sites, and the roles' loops have to stay resident in the SM's instruction cache.
@@ -161,7 +163,7 @@ struct Ctx {
     const uint32_t t0 = (uint32_t)clock();
     while (!mbar_try_wait(b, parity)) {
       if (*abort) return false;
-      if ((uint32_t)clock() - t0 > kTimeoutCycles) { *abort = code; return false; }
+      if ((uint32_t)clock() - t0 > budget) { *abort = code; return false; }
     }
     return true;
   }
@@ -484,7 +486,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   volatile int* misc = reinterpret_cast<volatile int*>(smem + kOffMisc);   // [0] tmem base, [1] abort flag
-  Ctx cx{sbase + kOffBar, misc + 1};
+  Ctx cx{sbase + kOffBar, misc + 1, p.wait_budget};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   KVQ_TRACE_DECL;
@@ -1045,15 +1047,17 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 int get_encode_fn(EncodeTiledFn* fn) {
-  static EncodeTiledFn cached = nullptr;
-  if (!cached) {
+  static std::atomic<EncodeTiledFn> cached{nullptr};     // a driver entry point: the same for every device
+  EncodeTiledFn f = cached.load(std::memory_order_acquire);
+  if (!f) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     KVQ_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres));
     if (qres != cudaDriverEntryPointSuccess || !sym) return record_cuda_error(cudaErrorSymbolNotFound);
-    cached = reinterpret_cast<EncodeTiledFn>(sym);
+    f = reinterpret_cast<EncodeTiledFn>(sym);
+    cached.store(f, std::memory_order_release);
   }
-  *fn = cached;
+  *fn = f;
   return KVQ_OK;
 }
 
@@ -1076,15 +1080,11 @@ int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, kvq_strides s
   return KVQ_OK;
 }
 
+// SM count of the current device; 148 (a B200) if the device cannot be asked: only sizes and launch counts
+// reported before a launch depend on it, and the launch itself fails loudly on such a device.
 int num_sms() {
-  static int cached = 0;
-  if (!cached) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-    cached = n;
-  }
-  return cached;
+  int n = 0;
+  return device_sm_count(&n) == KVQ_OK ? n : 148;
 }
 
 // Grid policy: how many CTAs, and how many leading units are computed whole (the rest are split).
@@ -1114,10 +1114,12 @@ Plan plan_grid(int64_t n_units, int64_t tiles) {
 template <int BITS, int GROUP>
 int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk, const CUtensorMap& mv, const TParams& p,
            const RotParams& rp, dim3 grid, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static PerDevice configured;                       // the attribute is per device
+  int dev = 0;
+  { const int r = current_device(&dev); if (r != KVQ_OK) return r; }
+  if (configured.first(dev)) {
     KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_tcgen05_kernel<BITS, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    configured = true;
+    configured.done(dev);
   }
   if (rp.qr) {                      // there are cached keys: rotate the query chunk first
     rotate_query_kernel<BITS, GROUP><<<dim3((unsigned)((rp.m_tokens + 15) / 16), (unsigned)(p.n_units / p.q_blocks)), 256, 0, st>>>(rp);
@@ -1170,6 +1172,9 @@ int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int
   return 1 + (cache_len > 0 ? 1 : 0) + (pl.n_whole != nu ? 1 : 0);   // attention, query pre-pass, merge
 }
 
+static std::atomic<uint32_t> g_wait_budget{0};           // 0: the default, kTimeoutCycles
+void set_attn_wait_budget(uint32_t cycles) { g_wait_budget.store(cycles, std::memory_order_relaxed); }
+
 // Common tail of both entry points.  `rot_area` (rot_area_bytes() bytes, 256-byte aligned; null only when
 // there are no cached keys) receives the rotated queries; `slots` holds the partial results of split units.
 static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, uint8_t* slots) {
@@ -1208,6 +1213,7 @@ static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t
   p.scale_log2 = a.softmax_scale * kLog2e;
   p.ax_coef = -a.softmax_scale / 24.0f;
   p.lse = a.lse; p.cached_mass = a.cached_mass; p.status = a.status_word;
+  { const uint32_t b = g_wait_budget.load(std::memory_order_relaxed); p.wait_budget = b ? b : kTimeoutCycles; }
   p.q_blocks = (int)qb; p.n_units = (int)nu; p.tiles = (int)tiles;
   p.partial = slots;
   p.ax_rows = rp.ax;
@@ -1238,8 +1244,7 @@ int launch_attn_tcgen05(const AttnArgs& a) {
 // ---- variant with built-in scratch ---------------------------------------------------------------
 //
 // Some callers may not allocate device memory at all (an inference server that hands its whole memory pool
-// to a framework allocator up front, code running while a CUDA graph is being captured, a plug-in that is
-// only given input and output pointers).  For them the split-unit path can run on a scratch buffer that is
+// to a framework allocator up front, a plug-in that is only given input and output pointers).  For them the split-unit path can run on a scratch buffer that is
 // part of the library image: every GPU that loads libkvq.so carries these 6.3 MiB until the process exits.
 // Layout: the rotated-query area for up to kStaticMaxRows query rows (batch * heads * m_tokens), then two
 // partial results for each of up to kStaticMaxCtas CTAs.
@@ -1253,18 +1258,18 @@ static __device__ __align__(256) uint8_t g_static_scratch[kStaticRotBytes + (siz
 // The array's name is only a host-side handle; the device address has to be asked for, once per device,
 // with that device current.
 static int static_scratch_ptr(uint8_t** out) {
-  constexpr int kMaxDevices = 64;
-  static uint8_t* ptrs[kMaxDevices] = {};
+  static std::atomic<uint8_t*> ptrs[kMaxDevices] = {};
   int dev = 0;
-  KVQ_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return KVQ_ERR_UNSUPPORTED;
-  if (!ptrs[dev]) {
+  { const int r = current_device(&dev); if (r != KVQ_OK) return r; }
+  uint8_t* ptr = ptrs[dev].load(std::memory_order_acquire);
+  if (!ptr) {
     void* p = nullptr;
     KVQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
     if (!p) return record_cuda_error(cudaErrorInvalidSymbol);
-    ptrs[dev] = static_cast<uint8_t*>(p);
+    ptr = static_cast<uint8_t*>(p);
+    ptrs[dev].store(ptr, std::memory_order_release);
   }
-  *out = ptrs[dev];
+  *out = ptr;
   return KVQ_OK;
 }
 

@@ -10,6 +10,27 @@ int record_cuda_error(cudaError_t e) {
   return KVQ_ERR_CUDA;
 }
 
+int current_device(int* dev) {
+  KVQ_CUDA_TRY(cudaGetDevice(dev));
+  if (*dev < 0 || *dev >= kMaxDevices) return KVQ_ERR_UNSUPPORTED;
+  return KVQ_OK;
+}
+
+int device_sm_count(int* sms) {
+  static std::atomic<int> cache[kMaxDevices] = {};
+  int dev = 0;
+  const int r = current_device(&dev);
+  if (r != KVQ_OK) return r;
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    KVQ_CUDA_TRY(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+    if (n <= 0) return record_cuda_error(cudaErrorInvalidDevice);
+    cache[dev].store(n, std::memory_order_relaxed);
+  }
+  *sms = n;
+  return KVQ_OK;
+}
+
 int check_shape(const kvq_cache_desc* d) {
   if (!d) return KVQ_ERR_INVALID_ARG;
   if (d->batch <= 0 || d->heads <= 0 || d->head_dim <= 0 || d->group <= 0 || d->capacity <= 0)
@@ -132,6 +153,14 @@ const char* kvq_status_string(int status) {
     case KVQ_ERR_WORKSPACE: return "workspace missing or too small";
     default: return "unknown status";
   }
+}
+
+int kvq_status_word_result(int32_t word) { return word == 0 ? KVQ_OK : KVQ_ERR_TIMEOUT; }
+
+int kvq_set_wait_budget_cycles(uint64_t cycles) {
+  if (cycles > 0xFFFF0000ull) return KVQ_ERR_INVALID_ARG;     // waits compare 32-bit clock differences
+  set_attn_wait_budget((uint32_t)cycles);
+  return KVQ_OK;
 }
 
 int kvq_cache_bytes(const kvq_cache_desc* desc, size_t out_bytes[6]) {

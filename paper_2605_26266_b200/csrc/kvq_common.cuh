@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "kvq.h"
 
 namespace kvq {
@@ -16,6 +18,22 @@ int record_cuda_error(cudaError_t e);
     cudaError_t kvq_e_ = (expr);                             \
     if (kvq_e_ != cudaSuccess) return ::kvq::record_cuda_error(kvq_e_); \
   } while (0)
+
+// Per-device host state.  One process may drive several GPUs, and several threads may call into the library:
+// whatever is looked up or configured once is kept per device ordinal, in atomics (a race only repeats an
+// idempotent CUDA call).
+constexpr int kMaxDevices = 64;
+// Ordinal of the calling thread's current device; KVQ_ERR_UNSUPPORTED beyond kMaxDevices.
+int current_device(int* dev);
+// Multiprocessor count of the current device (looked up once per device).
+int device_sm_count(int* sms);
+// "Has this been set up on the current device?" for one kernel instantiation: declare one static PerDevice per
+// instantiation; first() is true until done() has been called on that device.
+struct PerDevice {
+  std::atomic<unsigned char> flag[kMaxDevices] = {};
+  bool first(int dev) const { return flag[dev].load(std::memory_order_acquire) == 0; }
+  void done(int dev) { flag[dev].store(1, std::memory_order_release); }
+};
 
 // Shape part of the descriptor check (no pointers).
 int check_shape(const kvq_cache_desc* d);
@@ -56,6 +74,8 @@ bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_
 size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
 int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
 int launch_attn_tcgen05(const AttnArgs& a);
+// Cycle budget of the tcgen05 kernel's device-side waits for later launches (0 = the default of about a second).
+void set_attn_wait_budget(uint32_t cycles);
 // Same kernel, partial results of split units in the library's built-in scratch buffer (no caller workspace).
 int launch_attn_tcgen05_static(const AttnArgs& a);
 

@@ -377,12 +377,8 @@ int launch_quantize_append(const kvq_cache_desc* d, int64_t cache_len, const voi
   p.zero[0] = static_cast<uint16_t*>(d->k_zero); p.zero[1] = static_cast<uint16_t*>(d->v_zero);
   p.tiles_per_bh = (int)((n_tokens + kTileTokens - 1) / kTileTokens);
   p.total_tiles = (int64_t)d->batch * d->heads * p.tiles_per_bh;
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    sms = n;
-  }
+  int sms = 0;
+  { const int r = device_sm_count(&sms); if (r != KVQ_OK) return r; }
   const int64_t blocks = p.total_tiles < (int64_t)sms * kCtasPerSm ? p.total_tiles : (int64_t)sms * kCtasPerSm;
   dim3 grid((unsigned)blocks), block(kWarps * 32);
   if (p.total_tiles > 0x7FFFFFFFLL - 65536) return KVQ_ERR_UNSUPPORTED;

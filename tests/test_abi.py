@@ -106,3 +106,12 @@ def test_ring_cache_argument_rules_without_gpu(binding):
     unknown = b.kvq_cache_desc(1, 2, 128, 2, 32, 16, 256)
     sizes = (C.c_size_t * 6)()
     assert b.lib.kvq_cache_bytes(C.byref(unknown), sizes) == b.KVQ_ERR_INVALID_ARG
+
+
+def test_wait_budget_argument_and_status_word_mapping(binding):
+    b = binding
+    assert b.lib.kvq_set_wait_budget_cycles(0xFFFF0001) == b.KVQ_ERR_INVALID_ARG
+    assert b.lib.kvq_set_wait_budget_cycles(0) == b.KVQ_OK
+    assert b.kvq_status_word_result(0) == b.KVQ_OK
+    for word in (100, 204, 301, 404, -1):
+        assert b.kvq_status_word_result(word) == b.KVQ_ERR_TIMEOUT
