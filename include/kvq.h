@@ -171,7 +171,9 @@ int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len,
  *
  * q: [batch,heads,m_tokens,head_dim] strides q_strides; k_cur, v_cur: [batch,heads,n_cur,head_dim]
  * strides kv_strides; out: strides o_strides.  All device BF16, 16-byte aligned, strides
- * multiples of 8 elements.  cache_begin must be a multiple of 16 and
+ * multiples of 8 elements.  A batch or head stride of 0 (a chunk shared by all heads) is accepted: the tcgen05
+ * kernel cannot address such a tensor, so KVQ_KERNEL_AUTO runs the warp-level kernel for it and a forced
+ * KVQ_KERNEL_TCGEN05 returns KVQ_ERR_UNSUPPORTED.  cache_begin must be a multiple of 16 and
  * cache_begin + cache_len <= capacity.  cache_len == 0 is legal (plain attention over the
  * current chunk); n_cur must be >= 1; m_tokens == 0 is a no-op.
  *

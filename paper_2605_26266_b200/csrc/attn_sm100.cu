@@ -1061,16 +1061,25 @@ int get_encode_fn(EncodeTiledFn* fn) {
   return KVQ_OK;
 }
 
+// Byte strides of a [batch, heads, tokens, 128] BF16 tensor as a tensor map wants them: non-zero multiples of 16
+// below 2^40.  A size-1 dimension may come with any stride and gets a harmless valid one.  False if a real
+// dimension's stride cannot be encoded (0, as in a tensor expanded over heads, or too large).
+bool map_strides(kvq_strides s, int64_t tokens, int heads, int batch, cuuint64_t out[3]) {
+  const cuuint64_t st = tokens > 1 ? (cuuint64_t)s.t * 2 : (cuuint64_t)kD * 2;
+  const cuuint64_t sh = heads > 1 ? (cuuint64_t)s.h * 2 : st * (cuuint64_t)tokens;
+  const cuuint64_t sb = batch > 1 ? (cuuint64_t)s.b * 2 : sh * (cuuint64_t)heads;
+  out[0] = st; out[1] = sh; out[2] = sb;
+  if (s.t < 0 || s.h < 0 || s.b < 0) return false;
+  for (int i = 0; i < 3; ++i)
+    if (out[i] == 0 || out[i] % 16 != 0 || out[i] >= (1ull << 40)) return false;
+  return true;
+}
+
 // [batch, heads, tokens, 128] BF16 tensor -> 4-D map with a 64-column x 128-row box, 128-byte swizzle.
 int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, kvq_strides s, int64_t tokens, int heads, int batch) {
   cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)batch};
-  // a size-1 dimension may come with any stride; give it a harmless valid one
-  const cuuint64_t st = (cuuint64_t)s.t * 2;
-  const cuuint64_t sh = heads > 1 ? (cuuint64_t)s.h * 2 : st * (cuuint64_t)tokens;
-  const cuuint64_t sb = batch > 1 ? (cuuint64_t)s.b * 2 : sh * (cuuint64_t)heads;
-  cuuint64_t strides[3] = {st, sh, sb};
-  for (cuuint64_t v : strides)
-    if (v == 0 || v % 16 != 0 || v >= (1ull << 40)) return KVQ_ERR_UNSUPPORTED;
+  cuuint64_t strides[3];
+  if (!map_strides(s, tokens, heads, batch, strides)) return KVQ_ERR_UNSUPPORTED;
   cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -1138,6 +1147,13 @@ int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk,
 
 bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur) {
   return d->head_dim == kD && m_tokens >= 1 && n_cur >= 1;
+}
+
+bool attn_tcgen05_addressable(const AttnArgs& a) {
+  cuuint64_t st[3];
+  return map_strides(a.qs, a.m_tokens, a.desc->heads, a.desc->batch, st) &&
+         map_strides(a.kvs, a.n_cur, a.desc->heads, a.desc->batch, st) &&
+         map_strides(a.vs, a.n_cur, a.desc->heads, a.desc->batch, st);
 }
 
 static void schedule_shape(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur,

@@ -224,8 +224,17 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
                           out_bf16, o_strides, softmax_scale, flags);
   if (r != KVQ_OK) return r;
   int err;
-  const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
+  bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
+  AttnArgs a = make_attn_args(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens, n_cur,
+                              out_bf16, o_strides, softmax_scale, flags, lse_out, cached_mass_out, workspace,
+                              workspace_bytes, status_word, stream);
+  // Tensors TMA cannot address (a stride of 0, as in a chunk expanded over heads) go to the warp-level kernel,
+  // which takes any stride; a forced tcgen05 kernel fails here, before anything is launched.
+  if (tc && m_tokens > 0 && !attn_tcgen05_addressable(a)) {
+    if ((flags & KVQ_KERNEL_MASK) == KVQ_KERNEL_TCGEN05) return KVQ_ERR_UNSUPPORTED;
+    tc = false;
+  }
   const size_t rotv = rotv_bytes(desc, cache_len, m_tokens, n_cur);
   {
     const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0);
@@ -235,9 +244,6 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
     }
   }
   if (m_tokens == 0) return KVQ_OK;
-  AttnArgs a = make_attn_args(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens, n_cur,
-                              out_bf16, o_strides, softmax_scale, flags, lse_out, cached_mass_out, workspace,
-                              workspace_bytes, status_word, stream);
   if (rotv) {
     // values are cached rotated: bring the current chunk's values into the same space, attend, rotate the output back
     const kvq_strides dense{(int64_t)desc->heads * n_cur * desc->head_dim, n_cur * (int64_t)desc->head_dim, (int64_t)desc->head_dim};
@@ -266,6 +272,7 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
   const AttnArgs a = make_attn_args(desc, cache_begin, cache_len, q, q_strides, k_cur, v_cur, kv_strides, m_tokens,
                                     n_cur, out_bf16, o_strides, softmax_scale, flags, lse_out, cached_mass_out,
                                     nullptr, 0, status_word, stream);
+  if (!attn_tcgen05_addressable(a)) return KVQ_ERR_UNSUPPORTED;
   return launch_attn_tcgen05_static(a);
 }
 

@@ -71,6 +71,8 @@ int launch_rotate_rows(const kvq_cache_desc* d, const void* src, kvq_strides ss,
                        int64_t tokens, bool inverse, cudaStream_t st);
 // tcgen05 kernel: returns KVQ_ERR_UNSUPPORTED for shapes it does not cover.
 bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur);
+// Can TMA address the call's Q, K_cur, V_cur (no zero stride in a real dimension, byte strides below 2^40)?
+bool attn_tcgen05_addressable(const AttnArgs& a);
 size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
 int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
 int launch_attn_tcgen05(const AttnArgs& a);

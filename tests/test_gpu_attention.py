@@ -206,18 +206,59 @@ def test_sweep_config_full_rows(B, name, seed):
     _compare(B, g, o, n, q, kc, vc, T.sigma_of(w.head_dim), sel)
 
 
-@pytest.mark.parametrize("name,units", [("dit", [(0, 2), (0, 23)]), ("long", [(0, 13)]), ("prefix", [(0, 5), (0, 31)])])
-def test_large_configs_sampled_rows(B, name, units):
-    """Full-size launch; oracle on sampled rows touching every 128-row tile, for a few heads."""
+@pytest.mark.parametrize("name", ["dit", "long", "prefix"])
+def test_large_configs_every_head(B, name):
+    """Full-size launch, in the configuration bench.py times; the oracle on EVERY head, on rows that touch every
+    128-row tile (first, middle, last row of each, the ragged tail included) plus a few random ones.  The
+    oracle works head by head on host threads (one oracle cache per head), so its time stays in seconds."""
+    import concurrent.futures as cf
     w = inputs.WORKLOADS[name]
-    g, o, n, sel = _build(B, w, w.cached_chunks, units=units)
-    q, kc, vc = inputs.make_chunk(w, w.cached_chunks)
-    rows = inputs.sample_rows(w.chunk, 128, 32, seed=w.cfg_id)
-    _compare(B, g, o, n, q, kc, vc, T.sigma_of(w.head_dim), sel, rows=rows)
+    heads = [(b, h) for b in range(w.batch) for h in range(w.heads)]
+    g = B.Cache(w.batch, w.heads, w.head_dim, w.bits, w.group, w.capacity)
+    caches = [O.Cache(1, 1, w.head_dim, w.bits, w.group, w.capacity) for _ in heads]
+    one = lambda a, u: a[u[0]:u[0] + 1, u[1]:u[1] + 1]
+    n = 0
+    with cf.ThreadPoolExecutor(max_workers=16) as pool:
+        for c in range(w.cached_chunks):
+            _, k, v = inputs.make_chunk(w, c, need_q=False)
+            B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
+            lens = list(pool.map(lambda i: O.quantize_append(caches[i], n, one(k, heads[i]), one(v, heads[i])), range(len(heads))))
+            n = lens[0]
+        q, kc, vc = inputs.make_chunk(w, w.cached_chunks)
+        rows = inputs.sample_rows(w.chunk, 128, 8, seed=w.cfg_id)
+        sigma = T.sigma_of(w.head_dim)
+        qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+        lse = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
+        mass = torch.zeros_like(lse)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05, cache_len=n,
+                                   lse=lse, cached_mass=mass, status_word=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got, lse_h, mass_h = T.from_dev_bf16(out), lse.cpu().numpy().astype(np.float64), mass.cpu().numpy().astype(np.float64)
+        want = list(pool.map(lambda i: O.attn_corrected(caches[i], 0, n, one(q, heads[i]), one(kc, heads[i]),
+                                                         one(vc, heads[i]), sigma, correction=True, rows=rows),
+                             range(len(heads))))
+    worst = (0.0, 0.0)
+    for (b, h), wnt in zip(heads, want):
+        rel, mx = T.assert_attn_close(got[b, h][rows], wnt["out"][0], f"{name} head ({b},{h})")
+        worst = (max(worst[0], rel), max(worst[1], mx))
+        assert np.abs(lse_h[b, h][rows] - wnt["lse"][0]).max() < 2e-2, (b, h)
+        assert np.abs(mass_h[b, h][rows] - wnt["cached_mass"][0]).max() < 1e-2, (b, h)
+    print(f"{name}: worst rel-L2 {worst[0]:.2e}, worst max-abs {worst[1]:.2e} over {len(heads)} heads x {len(rows)} rows")
+    # the correction-off kernel on two heads
+    out_off = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_OFF | B.KVQ_KERNEL_TCGEN05, cache_len=n)
+    got_off = T.from_dev_bf16(out_off)
+    for i in (0, len(heads) - 1):
+        b, h = heads[i]
+        wnt = O.attn_corrected(caches[i], 0, n, one(q, heads[i]), one(kc, heads[i]), one(vc, heads[i]), sigma,
+                               correction=False, rows=rows)
+        T.assert_attn_close(got_off[b, h][rows], wnt["out"][0], f"{name} head ({b},{h}) uncorrected")
 
 
 def test_pipeline_config_steps(B):
-    """Attend-then-append over successive chunks (steps 0, 1, 2 and 5 checked; step 0 has an empty cache)."""
+    """Attend-then-append over the 16 successive chunks; the attention is checked at steps 0, 1, 2, 5 and 15
+    (step 0 has an empty cache, step 15 is the shape bench.py times: 30 720 cached tokens)."""
     w = inputs.WORKLOADS["pipeline"]
     units = [(0, 0), (1, 20)]
     sel = lambda a: np.stack([a[b, h] for (b, h) in units])[None]
@@ -225,13 +266,37 @@ def test_pipeline_config_steps(B):
     o = O.Cache(1, len(units), w.head_dim, w.bits, w.group, w.capacity)
     rows = inputs.sample_rows(w.chunk, 128, 16, seed=5)
     n = 0
-    for step in range(6):
-        q, k, v = inputs.make_chunk(w, step)
-        if step in (0, 1, 2, 5):
-            _compare(B, g, o, n, q, k, v, T.sigma_of(w.head_dim), sel, rows=rows)
-        B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
-        n = O.quantize_append(o, n, sel(k), sel(v))
+    for step in range(16):
+        check = step in (0, 1, 2, 5, 15)
+        q, k, v = inputs.make_chunk(w, step, need_q=check)
+        if check:
+            _compare(B, g, o, n, q, k, v, T.sigma_of(w.head_dim), sel, rows=rows,
+                     flags_list=None if step < 15 else [("tcgen05", B.KVQ_KERNEL_TCGEN05)])
+        if step < 15:
+            B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
+            n = O.quantize_append(o, n, sel(k), sel(v))
+    assert n == 15 * w.chunk
     T.assert_cache_equal(T.gpu_cache_arrays(g, n), o, n, units=units)
+
+
+def test_chunk_shared_by_all_heads_goes_to_the_warp_level_kernel(B):
+    """K_cur / V_cur with a head stride of 0 (one chunk expanded over the heads): TMA cannot address that, so the
+    automatic choice is the warp-level kernel, and forcing the tcgen05 kernel is refused before any launch."""
+    w = inputs.Workload("shared", 340, 1, 3, 128, 150, 0, 2, 64, 0, k_outliers=2, k_outlier_scale=4.0)
+    g, o, n, sel = _build(B, w, 2, tokens=140, cap=384)
+    q, kc, vc = inputs.make_chunk(w, 5)
+    kc[:] = kc[:, :1]; vc[:] = vc[:, :1]                     # every head sees head 0's chunk
+    qd = T.to_dev(q)
+    kd = T.to_dev(kc[:, :1]).expand(1, 3, 150, 128)
+    vd = T.to_dev(vc[:, :1]).expand(1, 3, 150, 128)
+    assert kd.stride(1) == 0
+    sigma = T.sigma_of(128)
+    out = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON, cache_len=n)
+    want = O.attn_corrected(o, 0, n, q, kc, vc, sigma, correction=True)["out"]
+    T.assert_attn_close(T.from_dev_bf16(out), want, "expanded chunk")
+    with pytest.raises(B.KvqError) as e:
+        B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05, cache_len=n)
+    assert e.value.status == B.KVQ_ERR_UNSUPPORTED
 
 
 @pytest.mark.parametrize("d,bits,group,dist", [(128, 2, 32, "student_t3"), (128, 2, 128, "normal"), (64, 4, 64, "normal")])

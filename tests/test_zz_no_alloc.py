@@ -61,6 +61,33 @@ def test_matches_workspace_entry_point_on_two_calls_in_a_row(B):
             assert np.abs(mass_st - mass_ws).max() < 1e-2
 
 
+def test_against_the_oracle_with_the_cta_count_capped(B):
+    """2 units of about 158 key tiles: the planner wants about 79 CTAs, the built-in buffer holds the partial
+    results of 32, so this entry point runs a different split (longer ranges per CTA, both slots of a CTA in
+    use) from kvq_attn_corrected.  Checked against the workspace entry point and, independently, the oracle."""
+    from oracle import kvq_oracle as O
+    w = inputs.Workload("noalloc_cap", 470, 1, 2, 128, 200, 0, 2, 64, 7, k_outliers=2, k_outlier_scale=4.0)
+    chunks, tokens = 5, 4000
+    g = B.Cache(1, 2, 128, 2, 64, 20096)
+    o = O.Cache(1, 2, 128, 2, 64, 20096)
+    n = 0
+    for c in range(chunks):
+        _, k, v = inputs.make_chunk(w, c, tokens=tokens)
+        B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
+        n = O.quantize_append(o, n, k, v)
+    q, kc, vc = inputs.make_chunk(w, 90)
+    qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
+    # the workspace entry would use far more CTAs than the static buffer has slots for
+    assert B.kvq_attn_workspace_bytes(g, n, 200, 200, B.KVQ_CORRECTION_ON) > 2 * 200 * 272 + 2 * 32 * 68608
+    for corr, flags in ((True, B.KVQ_CORRECTION_ON), (False, B.KVQ_CORRECTION_OFF)):
+        (o_ws, lse_ws, mass_ws), (o_st, lse_st, mass_st) = _both(B, g, qd, kd, vd, flags)
+        T.assert_attn_close(o_st, o_ws, "static scratch vs workspace")
+        want = O.attn_corrected(o, 0, n, q, kc, vc, T.sigma_of(128), correction=corr)
+        T.assert_attn_close(o_st, want["out"], "static scratch vs oracle")
+        assert np.abs(lse_st - want["lse"]).max() < 2e-2
+        assert np.abs(mass_st - want["cached_mass"]).max() < 1e-2
+
+
 def test_unsplit_problem_uses_only_the_query_area_and_is_identical(B):
     g, q, kc, vc = _problem(B, heads=80, m=100, chunks=2, chunk_tokens=300, n_cur=256, seed=3)   # 80 units: one CTA each
     # no partial-result slots: the workspace is just the rotated queries (256 + 16 bytes per query row)
