@@ -15,6 +15,9 @@ What it follows (paper sections / equations):
 * Attention: Algorithm 1 (Taylor-corrected attention, group-wise), Eqs. (2)-(4)
   (scores, partition sums, cached mass), Eq. (15) / Eq. (25) (grouped Taylor
   correction, with the rotated query under QuaRot), Eq. (12) (exact sinh form).
+* Diagnostics: the Jensen-Shannon divergence between the attention weights over
+  all keys with the quantized (or corrected) cache and with the BF16 cache
+  (App. "Attention JSD Distributions").
 
 Readings of points the paper leaves open (each one is a reading, "parity
 unpinned" by the paper itself; the quantizer as a whole is pinned by the error
@@ -323,14 +326,16 @@ def exact_bias(q_rot, key_scale, group, sigma):
 
 def attn_corrected_head(q_bits, kcur_bits, vcur_bits, k_codes, k_scale, k_zero,
                         v_codes, v_scale, v_zero, bits, group, sigma, correction=True,
-                        rotate=True, signs=None, rows=None, exact=False, rotate_v=False, k_group=None):
+                        rotate=True, signs=None, rows=None, exact=False, rotate_v=False, k_group=None,
+                        return_weights=False):
     """One (batch, head) unit of Algorithm 1.
 
     q_bits [M, d], kcur_bits/vcur_bits [N_R, d] BF16 bit patterns; cache slices for
     the attended window, [N_S, ...].  rows: optional index array of query rows.
     Returns dict(out [m, d], lse [m], cached_mass [m], current_mass [m]); the two masses are
     P_S and P_R of Eq. (4), summed separately.  k_group: channels per key group if it differs from the values'
-    (1 for per-channel keys, whose k_scale / k_zero arrive expanded to one row per token, [N_S, d])."""
+    (1 for per-channel keys, whose k_scale / k_zero arrive expanded to one row per token, [N_S, d]).
+    return_weights: also return "weights" [m, N_S + N_R], the softmax rows themselves (cached keys first)."""
     k_group = group if k_group is None else k_group
     q = bf16_bits_to_f64(q_bits)
     if rows is not None:
@@ -366,8 +371,11 @@ def attn_corrected_head(q_bits, kcur_bits, vcur_bits, k_codes, k_scale, k_zero,
         if signs is not None:
             o_s = o_s * np.asarray(signs, dtype=np.float64)
     out = o_s + p[:, n_s:] @ vr
-    return {"out": out, "lse": (mx + np.log(z))[:, 0],
-            "cached_mass": p[:, :n_s].sum(axis=1), "current_mass": p[:, n_s:].sum(axis=1)}
+    res = {"out": out, "lse": (mx + np.log(z))[:, 0],
+           "cached_mass": p[:, :n_s].sum(axis=1), "current_mass": p[:, n_s:].sum(axis=1)}
+    if return_weights:
+        res["weights"] = p
+    return res
 
 
 def attn_corrected(cache: Cache, cache_begin, cache_len, q_bits, kcur_bits, vcur_bits,
@@ -396,6 +404,55 @@ def attn_corrected(cache: Cache, cache_begin, cache_len, q_bits, kcur_bits, vcur
         cmasses.append(r["current_mass"])
     return {"out": np.stack(outs), "lse": np.stack(lses), "cached_mass": np.stack(masses),
             "current_mass": np.stack(cmasses)}
+
+
+def attention_weights_bf16(q_bits, k_bits, sigma, rows=None):
+    """softmax(sigma q k^T) row by row for BF16 q [M, d] and k [N, d]: the attention weights of the unquantized
+    (BF16) cache that the quantized ones are compared with."""
+    q = bf16_bits_to_f64(q_bits)
+    if rows is not None:
+        q = q[rows]
+    s = sigma * (q @ bf16_bits_to_f64(k_bits).T)
+    e = np.exp(s - s.max(axis=1, keepdims=True))
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def jsd_rows(p, r):
+    """Jensen-Shannon divergence of each row of p from the same row of r (natural logarithm, 0 log 0 = 0):
+    JSD = KL(p || m) / 2 + KL(r || m) / 2 with the mixture m = (p + r) / 2; between 0 and log 2."""
+    p = np.asarray(p, dtype=np.float64)
+    r = np.asarray(r, dtype=np.float64)
+    m = 0.5 * (p + r)
+
+    def kl(a):
+        t = np.zeros_like(a)
+        nz = a > 0
+        t[nz] = a[nz] * np.log(a[nz] / m[nz])
+        return t.sum(axis=-1)
+
+    return 0.5 * kl(p) + 0.5 * kl(r)
+
+
+def attn_weight_jsd(cache: Cache, cache_begin, cache_len, q_bits, kcur_bits, kcached_bits, sigma,
+                    correction=True, rows=None, heads=None):
+    """Per query row, the JSD between the attention weights over all keys [cached ; current] computed with the
+    quantized cache (Algorithm 1, with or without the correction) and with the BF16 keys `kcached_bits`
+    [B, H, cache_len, d] those cache entries were quantized from.  Returns [unit, row]."""
+    B, H = q_bits.shape[:2]
+    units = heads if heads is not None else [(b, h) for b in range(B) for h in range(H)]
+    sl = cache.slots(cache_begin, cache_len)
+    out = []
+    for (b, h) in units:
+        vz = np.zeros_like(kcur_bits[b, h])                # the weights do not depend on the values
+        wq = attn_corrected_head(
+            q_bits[b, h], kcur_bits[b, h], vz,
+            cache.k_codes[b, h, sl], cache.k_scale[b, h, sl], cache.k_zero[b, h, sl],
+            cache.v_codes[b, h, sl], cache.v_scale[b, h, sl], cache.v_zero[b, h, sl],
+            cache.bits, cache.group, sigma, correction, cache.rotate_k, cache.signs, rows,
+            return_weights=True)["weights"]
+        k_all = np.concatenate([kcached_bits[b, h], kcur_bits[b, h]], axis=0)
+        out.append(jsd_rows(wq, attention_weights_bf16(q_bits[b, h], k_all, sigma, rows)))
+    return np.stack(out)
 
 
 def effective_bits(bits, group):

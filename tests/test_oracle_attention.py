@@ -363,3 +363,74 @@ def test_per_channel_keys_bias_is_one_scalar_per_block_and_matches_app_e():
     want = p[:, :64] @ v_hat + p[:, 64:] @ f(vc)[0, 0]
     assert np.abs(got["out"][0] - want).max() < 1e-12
     assert np.abs(got["cached_mass"][0] - p[:, :64].sum(1)).max() < 1e-12
+
+
+# ---- attention-weight diagnostics: the Jensen-Shannon divergence of the appendix on attention JSD ----
+
+def test_jsd_closed_forms_and_library_routine():
+    import scipy.spatial.distance
+    ln2 = math.log(2.0)
+    p = np.array([[1.0, 0.0, 0.0], [0.5, 0.5, 0.0], [0.2, 0.3, 0.5]])
+    assert np.abs(O.jsd_rows(p, p)).max() == 0.0                         # a distribution against itself
+    assert abs(O.jsd_rows([[1.0, 0.0]], [[0.0, 1.0]])[0] - ln2) < 1e-15  # disjoint supports: the upper bound log 2
+    # (1/2, 1/2) against (1, 0): KL(p||m) = log 2 - (1/2) log 3 ... worked by hand: (3/4) log(4/3) - ... = below
+    want = 0.5 * (0.5 * math.log(0.5 / 0.75) + 0.5 * math.log(0.5 / 0.25)) + 0.5 * math.log(1.0 / 0.75)
+    assert abs(O.jsd_rows([[0.5, 0.5]], [[1.0, 0.0]])[0] - want) < 1e-15 and abs(want - 0.21576155433883565) < 1e-12
+    r = np.random.default_rng(5)
+    a = r.random((40, 17)); a /= a.sum(1, keepdims=True)
+    b = r.random((40, 17)); b[:, :3] = 0.0; b /= b.sum(1, keepdims=True)  # zeros: 0 log 0 = 0
+    got = O.jsd_rows(a, b)
+    lib = np.array([scipy.spatial.distance.jensenshannon(a[i], b[i]) ** 2 for i in range(40)])   # a distance: the square root
+    assert np.abs(got - lib).max() < 1e-14
+    assert np.abs(got - O.jsd_rows(b, a)).max() < 1e-15                  # symmetric
+    assert (got > 0).all() and (got < ln2).all()
+
+
+def test_bf16_reference_weights_are_the_library_softmax():
+    r = np.random.default_rng(6)
+    bf = lambda x: inputs.f32_to_bf16_bits(x.astype(np.float32))
+    q, k = bf(r.standard_normal((9, 64))), bf(r.standard_normal((21, 64)))
+    got = O.attention_weights_bf16(q, k, 0.2, rows=np.array([0, 4, 8]))
+    qt = torch.from_numpy(O.bf16_bits_to_f64(q))[[0, 4, 8]]
+    kt = torch.from_numpy(O.bf16_bits_to_f64(k))
+    want = torch.softmax(0.2 * qt @ kt.T, dim=-1).numpy()
+    assert np.abs(got - want).max() < 1e-15
+
+
+def test_returned_weights_are_the_rows_behind_output_and_mass():
+    q, kc, vc, ks, vs, cache = _tiny_problem(31, 64, 32, 2, 7, 4, 5)
+    sl = cache.slots(0, 7)
+    res = O.attn_corrected_head(q[0, 0], kc[0, 0], vc[0, 0], cache.k_codes[0, 0, sl], cache.k_scale[0, 0, sl],
+                                cache.k_zero[0, 0, sl], cache.v_codes[0, 0, sl], cache.v_scale[0, 0, sl],
+                                cache.v_zero[0, 0, sl], 2, 32, 0.125, return_weights=True)
+    w = res["weights"]
+    assert w.shape == (5, 11) and np.abs(w.sum(1) - 1).max() < 1e-14
+    assert np.abs(w[:, :7].sum(1) - res["cached_mass"]).max() < 1e-15
+    v_all = np.concatenate([O.dequant(cache.v_codes[0, 0, sl], cache.v_scale[0, 0, sl], cache.v_zero[0, 0, sl], 2, 32),
+                            O.bf16_bits_to_f64(vc[0, 0])])
+    assert np.abs(w @ v_all - res["out"]).max() < 1e-13
+
+
+def test_weight_jsd_vanishes_for_a_lossless_cache_and_not_otherwise():
+    # codes that reproduce the keys exactly, no rotation, no correction: the two weight vectors coincide
+    q, kc, vc, ks, vs, cache = _tiny_problem(32, 64, 32, 2, 9, 3, 4, rotate=False, lossless=True)
+    j = O.attn_weight_jsd(cache, 0, 9, q, kc, ks, 0.125, correction=False)
+    assert j.shape == (1, 4) and np.abs(j).max() < 1e-25
+    # the correction alone moves the weights (the steps are 0.5, not 0)
+    assert O.attn_weight_jsd(cache, 0, 9, q, kc, ks, 0.125, correction=True).min() > 1e-9
+    # a lossy cache: positive, below log 2, and equal to the definition written out for one row
+    q, kc, vc, ks, vs, cache = _tiny_problem(33, 64, 32, 2, 9, 3, 4)
+    j = O.attn_weight_jsd(cache, 0, 9, q, kc, ks, 0.125, correction=True, rows=np.array([2]))
+    assert 0 < j[0, 0] < math.log(2.0)
+    p = O.attn_corrected_head(q[0, 0], kc[0, 0], vc[0, 0], cache.k_codes[0, 0, :9], cache.k_scale[0, 0, :9],
+                              cache.k_zero[0, 0, :9], cache.v_codes[0, 0, :9], cache.v_scale[0, 0, :9],
+                              cache.v_zero[0, 0, :9], 2, 32, 0.125, rows=np.array([2]), return_weights=True)["weights"][0]
+    f = O.bf16_bits_to_f64
+    s = [0.125 * float(f(q)[0, 0, 2] @ kk) for kk in np.concatenate([f(ks)[0, 0], f(kc)[0, 0]])]
+    z = sum(math.exp(x) for x in s)
+    total = 0.0
+    for pi, si in zip(p, s):
+        ri = math.exp(si) / z
+        mi = 0.5 * (pi + ri)
+        total += 0.5 * pi * math.log(pi / mi) + 0.5 * ri * math.log(ri / mi)
+    assert abs(total - j[0, 0]) < 1e-15

@@ -70,6 +70,16 @@ MUTATIONS = [
     ("rotated values not rotated back", "        o_s = rotate_f64(o_s, None)\n", "        o_s = o_s + 0.0\n"),
     ("per-channel keys take the token's own row of steps", "ksl = sl // cache.group if cache.k_per_channel else sl",
      "ksl = sl % (cache.capacity // cache.group) if cache.k_per_channel else sl"),
+    # ---- attention-weight diagnostics
+    ("JSD without the halves", "return 0.5 * kl(p) + 0.5 * kl(r)", "return kl(p) + kl(r)"),
+    ("JSD one-sided", "return 0.5 * kl(p) + 0.5 * kl(r)", "return 0.5 * kl(p) + 0.5 * kl(p)"),
+    ("JSD mixture not halved", "m = 0.5 * (p + r)", "m = p + r"),
+    ("BF16 reference weights without the softmax scale", "s = sigma * (q @ bf16_bits_to_f64(k_bits).T)", "s = q @ bf16_bits_to_f64(k_bits).T"),
+    ("JSD reference keys in the wrong order", "k_all = np.concatenate([kcached_bits[b, h], kcur_bits[b, h]], axis=0)",
+     "k_all = np.concatenate([kcur_bits[b, h], kcached_bits[b, h]], axis=0)"),
+    ("weights returned unnormalised", '        res["weights"] = p', '        res["weights"] = e'),
+    ("JSD of the uncorrected weights only", "cache.bits, cache.group, sigma, correction, cache.rotate_k, cache.signs, rows,\n            return_weights=True)",
+     "cache.bits, cache.group, sigma, False, cache.rotate_k, cache.signs, rows,\n            return_weights=True)"),
     ("effective bits count 16 metadata bits", "return bits + 24.0 / group", "return bits + 16.0 / group"),
 ]
 
