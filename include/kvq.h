@@ -235,6 +235,27 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
                                       int32_t* status_word, kvq_stream_t stream);
 
 /*
+ * Attention-weight diagnostic (the paper's appendix "Attention JSD Distributions"): for every (batch, head) and
+ * query row, the Jensen-Shannon divergence (natural logarithm, between 0 and log 2) between
+ *   p = softmax over the scores s_i, s_r of kvq_attn_corrected (quantized cache, correction on or off), and
+ *   r = softmax over softmax_scale * q . k for the BF16 keys [k_cached_bf16 ; k_cur],
+ * both over all cache_len + n_cur keys.  k_cached_bf16 [batch, heads, cache_len, head_dim] (device BF16, strides
+ * kcached_strides) are the keys the cache window [cache_begin, cache_begin + cache_len) was quantized from: an
+ * analysis input that a deployment does not keep; may be NULL when cache_len is 0.
+ * jsd_out: device float [batch, heads, m_tokens].  Nothing of size m_tokens x keys is written: scores are
+ * recomputed in FP32 on the CUDA cores in two passes (log-sum-exps, then the divergence), so this is an
+ * analysis call, not a fast one.  flags: KVQ_CORRECTION_ON or KVQ_CORRECTION_OFF only; not for
+ * KVQ_K_PER_CHANNEL caches.  Errors: as kvq_attn_corrected's argument checks, KVQ_ERR_UNSUPPORTED for the
+ * options above, KVQ_ERR_CUDA.
+ */
+int kvq_attn_weight_jsd(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
+                        const void* q, kvq_strides q_strides,
+                        const void* k_cur, kvq_strides kcur_strides,
+                        const void* k_cached_bf16, kvq_strides kcached_strides,
+                        int64_t m_tokens, int64_t n_cur, float softmax_scale, uint32_t flags,
+                        float* jsd_out, kvq_stream_t stream);
+
+/*
  * Test aid: expand the packed codes of cache tokens [begin, begin + n) to one byte per element,
  * out_codes device u8 [batch, heads, n, head_dim], in canonical channel order (the order of
  * Eq. (1)'s vector x).  which: 0 = keys, 1 = values.

@@ -80,6 +80,10 @@ def _load():
     lib.kvq_status_word_result.argtypes = [C.c_int32]
     lib.kvq_set_wait_budget_cycles.restype = C.c_int
     lib.kvq_set_wait_budget_cycles.argtypes = [C.c_uint64]
+    lib.kvq_attn_weight_jsd.restype = C.c_int
+    lib.kvq_attn_weight_jsd.argtypes = [
+        C.POINTER(kvq_cache_desc), C.c_int64, C.c_int64, C.c_void_p, kvq_strides, C.c_void_p, kvq_strides,
+        C.c_void_p, kvq_strides, C.c_int64, C.c_int64, C.c_float, C.c_uint32, C.c_void_p, C.c_void_p]
     lib.kvq_unpack_codes.restype = C.c_int
     lib.kvq_unpack_codes.argtypes = [C.POINTER(kvq_cache_desc), C.c_int, C.c_int64, C.c_int64,
                                      C.c_void_p, C.c_void_p]
@@ -231,6 +235,24 @@ def kvq_attn_corrected_static_scratch(cache: Cache, q, k_cur, v_cur, softmax_sca
         C.byref(cache.desc), cache_begin, n_cache, q.data_ptr(), _strides(q), k_cur.data_ptr(), v_cur.data_ptr(),
         _strides(k_cur), q.shape[2], k_cur.shape[2], out.data_ptr(), _strides(out), float(softmax_scale), flags,
         _ptr(lse), _ptr(cached_mass), _ptr(status_word), _stream()), "kvq_attn_corrected_static_scratch")
+    return out
+
+
+def kvq_attn_weight_jsd(cache: Cache, q, k_cur, k_cached, softmax_scale, flags=KVQ_CORRECTION_ON, cache_begin=0,
+                        cache_len=None, out=None):
+    """Per-row JSD of the attention weights against those of the BF16 keys k_cached ([batch, heads, cache_len,
+    head_dim], the keys the attended cache window was quantized from); returns float32 [batch, heads, rows]."""
+    for t in (q, k_cur) + ((k_cached,) if k_cached is not None else ()):
+        assert t.dtype == torch.bfloat16 and t.is_cuda
+    n_cache = cache.length - cache_begin if cache_len is None else cache_len
+    assert n_cache == 0 or k_cached.shape[2] == n_cache
+    if out is None:
+        out = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    kc_ptr, kc_str = (k_cached.data_ptr(), _strides(k_cached)) if n_cache else (None, kvq_strides(0, 0, 0))
+    _check(lib.kvq_attn_weight_jsd(
+        C.byref(cache.desc), cache_begin, n_cache, q.data_ptr(), _strides(q), k_cur.data_ptr(), _strides(k_cur),
+        kc_ptr, kc_str, q.shape[2], k_cur.shape[2], float(softmax_scale), flags, out.data_ptr(), _stream()),
+        "kvq_attn_weight_jsd")
     return out
 
 

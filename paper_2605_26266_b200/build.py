@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libkvq.so")
-SOURCES = ["kvq_api.cu", "quantize_append.cu", "rotate_rows.cu", "attn_mma_sync.cu", "attn_sm100.cu"]
+SOURCES = ["kvq_api.cu", "quantize_append.cu", "rotate_rows.cu", "attn_mma_sync.cu", "attn_jsd.cu", "attn_sm100.cu"]
 HEADERS = [os.path.join(CSRC, "kvq_common.cuh"), os.path.join(ROOT, "include", "kvq.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -276,6 +276,27 @@ int kvq_attn_corrected_static_scratch(const kvq_cache_desc* desc, int64_t cache_
   return launch_attn_tcgen05_static(a);
 }
 
+int kvq_attn_weight_jsd(const kvq_cache_desc* desc, int64_t cache_begin, int64_t cache_len,
+                        const void* q, kvq_strides q_strides, const void* k_cur, kvq_strides kcur_strides,
+                        const void* k_cached_bf16, kvq_strides kcached_strides, int64_t m_tokens, int64_t n_cur,
+                        float softmax_scale, uint32_t flags, float* jsd_out, kvq_stream_t stream) {
+  int r = check_attn_args(desc, cache_begin, cache_len, m_tokens, n_cur, flags);
+  if (r != KVQ_OK) return r;
+  if ((r = check_desc(desc)) != KVQ_OK) return r;
+  if (flags & (KVQ_CORRECTION_EXACT | KVQ_KERNEL_MASK)) return KVQ_ERR_UNSUPPORTED;      // Taylor form or none; one kernel
+  if (desc->flags & KVQ_K_PER_CHANNEL) return KVQ_ERR_UNSUPPORTED;
+  if (!jsd_out) return KVQ_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 1e30f)) return KVQ_ERR_INVALID_ARG;
+  if ((r = check_tensor(q, q_strides)) != KVQ_OK) return r;
+  if ((r = check_tensor(k_cur, kcur_strides)) != KVQ_OK) return r;
+  if (cache_len > 0 && (r = check_tensor(k_cached_bf16, kcached_strides)) != KVQ_OK) return r;
+  if (m_tokens == 0) return KVQ_OK;
+  const AttnArgs a = make_attn_args(desc, cache_begin, cache_len, q, q_strides, k_cur, k_cur, kcur_strides, m_tokens,
+                                    n_cur, nullptr, q_strides, softmax_scale, flags, nullptr, nullptr, nullptr, 0,
+                                    nullptr, stream);
+  return launch_attn_jsd(a, k_cached_bf16, kcached_strides, jsd_out);
+}
+
 int kvq_unpack_codes(const kvq_cache_desc* desc, int which, int64_t begin, int64_t n,
                      uint8_t* out_codes, kvq_stream_t stream) {
   int r = check_desc(desc);

@@ -66,6 +66,8 @@ struct AttnArgs {
   cudaStream_t stream;
 };
 int launch_attn_mma_sync(const AttnArgs& a);
+// Per-row Jensen-Shannon divergence of the attention weights against those of the BF16 keys k_ref (analysis kernel).
+int launch_attn_jsd(const AttnArgs& a, const void* k_ref, kvq_strides ref_strides, float* jsd_out);
 // y = (1/sqrt d) H (signs . x) per row (inverse: x = signs . ((1/sqrt d) H y)), BF16 [batch, heads, tokens, head_dim]
 int launch_rotate_rows(const kvq_cache_desc* d, const void* src, kvq_strides ss, void* dst, kvq_strides ds,
                        int64_t tokens, bool inverse, cudaStream_t st);

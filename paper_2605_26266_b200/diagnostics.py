@@ -1,7 +1,7 @@
 """Attention-level diagnostics of Section 6 ("attention stealing"), on the GPU path.
 
-The cached-mass shift of Eq. (9), dP_S = P^_S - P_S, and the error of the attention output against the
-unquantized cache, with the correction off and on.  Everything heavy is a call of the C ABI (through the
+The cached-mass shift of Eq. (9), dP_S = P^_S - P_S, the Jensen-Shannon divergence of the attention weights
+and the error of the attention output against the unquantized cache, with the correction off and on.  Everything heavy is a call of the C ABI (through the
 binding): the quantized numbers are kvq_attn_corrected's `cached_mass_out` and output; the unquantized
 reference is the same kernel run with an empty cache window and the BF16 cached keys/values passed as part of
 the "current chunk", where P_S follows from two log-sum-exps (all keys, current keys only).  What is left
@@ -23,8 +23,9 @@ def attention_stealing(cache: "B.Cache", k_cached, v_cached, q, k_cur, v_cur, so
     """k_cached, v_cached: the BF16 tensors [batch, heads, n, head_dim] whose quantized form is the window
     [cache_begin, cache_begin + n) of `cache`.  Returns a dict of per-row tensors [batch, heads, rows]:
     `p_s_ref`, `p_s_uncorrected`, `p_s_corrected`, `p_s_exact` (Taylor correction of Eq. (15), exact one of
-    Eq. (12)), their differences to the reference `dps_*` (Eq. (9)), and `mse_*` (mean squared error of the
-    output rows against the unquantized cache)."""
+    Eq. (12)), their differences to the reference `dps_*` (Eq. (9)), `mse_*` (mean squared error of the
+    output rows against the unquantized cache) and `jsd_uncorrected`, `jsd_corrected` (divergence of the attention
+    weights over all keys from those of the unquantized cache, kvq_attn_weight_jsd)."""
     n = k_cached.shape[2]
     n_cache = n if cache_len is None else cache_len
     assert n_cache == n, "the BF16 copy must cover exactly the attended window"
@@ -54,6 +55,9 @@ def attention_stealing(cache: "B.Cache", k_cached, v_cached, q, k_cur, v_cur, so
         res["p_s_" + name] = mass
         res["dps_" + name] = mass - p_s_ref
         res["mse_" + name] = (out.float() - out_ref.float()).pow(2).mean(dim=-1)
+        if flag != B.KVQ_CORRECTION_EXACT and not (cache.desc.flags & B.KVQ_K_PER_CHANNEL):
+            res["jsd_" + name] = B.kvq_attn_weight_jsd(cache, q, k_cur, k_cached, softmax_scale, flag,
+                                                       cache_begin=cache_begin, cache_len=n_cache)
     return res
 
 
