@@ -9,7 +9,9 @@
 // reproducible bit for bit.  A CTA stages the packed bytes of 32 consecutive tokens in shared memory and
 // writes them out with 128-bit stores (tokens of one (batch, head) are contiguous in the cache).  CTAs are
 // persistent (a few per SM) and keep the next tile's loads in flight while they work on the current one.
-// By its bytes the kernel is HBM-bound on its BF16 input.
+// By its bytes the kernel would be HBM-bound on its BF16 input; in fact it is bound by instruction issue: the
+// bit-exact contract fixes one IEEE operation per butterfly, division, rounding and clamp, about 230 warp
+// instructions per token-head, against 576 bytes.
 #include "kvq_common.cuh"
 
 namespace kvq {
@@ -72,9 +74,12 @@ __device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int l8, in
   constexpr int lanes_per_group = GROUP / EPL;
   constexpr int G = (8 * EPL) / GROUP;
 
-  float mn = x[0], mx = x[0];
+  float mn = fminf(x[0], x[1]), mx = fmaxf(x[0], x[1]);
 #pragma unroll
-  for (int e = 1; e < EPL; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+  for (int e = 2; e < EPL; e += 2) {                  // three-input minimum and maximum: one instruction per two elements
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(mn) : "f"(mn), "f"(x[e]), "f"(x[e + 1]));
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(mx) : "f"(mx), "f"(x[e]), "f"(x[e + 1]));
+  }
 #pragma unroll
   for (int off = 1; off < lanes_per_group; off *= 2) {
     mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
@@ -113,11 +118,23 @@ __device__ __forceinline__ void quantize_stage(const float (&x)[EPL], int l8, in
 #pragma unroll
   for (int k = 0; k < kChunks; ++k) acc[k] = 8388608.f;
   if (!slow) {
+    // q + 1.5*2^23 is 1.5*2^23 + rint(q); taking off 1.5*2^23 - zero (an integer below 2^24, so exact) leaves
+    // rint(q) + zero, the sum Eq. (1) clamps.  While the zero-point is exact in BF16 (|zero| <= 256) the sum cannot
+    // be negative (x >= min and both roundings are monotonic), so the lower clamp is only taken when some group of
+    // the warp has a rounded zero-point.
+    const float kz = __fsub_rn(kRound, zs);
+    if (__any_sync(0xFFFFFFFFu, zs != z)) {
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const float r = __fsub_rn(__fadd_rn(fast_div(x[e], ds, rds), kRound), kRound);
-      const float c = fminf(fmaxf(__fadd_rn(r, zs), 0.0f), L);
-      acc[(e * BITS) / 16] = __fmaf_rn(c, (float)(1u << ((e * BITS) % 16)), acc[(e * BITS) / 16]);
+      for (int e = 0; e < EPL; ++e) {
+        const float c = fminf(fmaxf(__fsub_rn(__fadd_rn(fast_div(x[e], ds, rds), kRound), kz), 0.0f), L);
+        acc[(e * BITS) / 16] = __fmaf_rn(c, (float)(1u << ((e * BITS) % 16)), acc[(e * BITS) / 16]);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        const float c = fminf(__fsub_rn(__fadd_rn(fast_div(x[e], ds, rds), kRound), kz), L);
+        acc[(e * BITS) / 16] = __fmaf_rn(c, (float)(1u << ((e * BITS) % 16)), acc[(e * BITS) / 16]);
+      }
     }
   } else {
 #pragma unroll
