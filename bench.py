@@ -38,7 +38,7 @@ L2_FLUSH_BYTES = 512 << 20
 MIN_REGION_MS = 120.0          # every leg's timed region is at least this long (the clock sampler polls every 50 ms)
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of attn_tcgen05_kernel, from the ncu captures
-# summarised under profiles/ (the file named there gives the command and the commit it was taken at)
+# summarised under profiles/ (launches_bench_long.md gives the commands; the figures go stale when the kernel changes)
 NCU_TRAFFIC_BYTES = {}
 try:
     with open(os.path.join(ROOT, "profiles", "traffic.json")) as _f:
