@@ -84,6 +84,9 @@ extern "C" {
 #define KVQ_KERNEL_AUTO       0u
 #define KVQ_KERNEL_MMA_SYNC   (1u << 8)  /* force the warp-level mma.sync kernel (cross-check / fallback shapes) */
 #define KVQ_KERNEL_TCGEN05    (2u << 8)  /* force the tcgen05/TMEM kernel; KVQ_ERR_UNSUPPORTED if the shape is not covered */
+#define KVQ_KERNEL_TCGEN05_PAIR (3u << 8) /* the tcgen05 kernel on pairs of SMs (thread-block clusters of two CTAs that share
+                                            one tcgen05.mma of 256 rows): each CTA of a pair expands only half of every
+                                            cached key and value tile.  Same results; same shapes as KVQ_KERNEL_TCGEN05 */
 #define KVQ_KERNEL_MASK       (3u << 8)
 
 typedef void* kvq_stream_t;          /* a cudaStream_t */

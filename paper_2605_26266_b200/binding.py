@@ -24,7 +24,7 @@ KVQ_RING = 2
 KVQ_ROTATE_V = 4
 KVQ_K_PER_CHANNEL = 8
 KVQ_CORRECTION_OFF, KVQ_CORRECTION_ON, KVQ_CORRECTION_EXACT = 0, 1, 2
-KVQ_KERNEL_AUTO, KVQ_KERNEL_MMA_SYNC, KVQ_KERNEL_TCGEN05 = 0, 1 << 8, 2 << 8
+KVQ_KERNEL_AUTO, KVQ_KERNEL_MMA_SYNC, KVQ_KERNEL_TCGEN05, KVQ_KERNEL_TCGEN05_PAIR = 0, 1 << 8, 2 << 8, 3 << 8
 
 
 class kvq_cache_desc(C.Structure):

@@ -245,18 +245,20 @@ struct Raw {   // packed codes and metadata of one cached token (keys or values)
   uint32_t z01, z23;     // zero-points (BF16 bits) of up to 4 groups
 };
 
-template <int BITS, int G>
+// Loads NW code words of the token, starting at word `word0` (a multiple of 4), into r.w[0 .. NW), and the token's
+// metadata.  NW is the whole row, or half of it for a CTA of a pair.
+template <int BITS, int G, int NW = Raw<BITS>::kWords>
 __device__ __forceinline__ void load_raw(Raw<BITS>& r, const uint8_t* codes, const uint8_t* scale, const uint16_t* zero,
-                                         int64_t tok, bool valid) {
+                                         int64_t tok, bool valid, int word0 = 0) {
   if (!valid) {   // rows past the end of the cache dequantize to exact zeros
 #pragma unroll
-    for (int i = 0; i < Raw<BITS>::kWords; ++i) r.w[i] = 0;
+    for (int i = 0; i < NW; ++i) r.w[i] = 0;
     r.sbytes = 0; r.z01 = 0; r.z23 = 0;
     return;
   }
-  const uint4* cw = reinterpret_cast<const uint4*>(codes + tok * (kD * BITS / 8));
+  const uint4* cw = reinterpret_cast<const uint4*>(codes + tok * (kD * BITS / 8)) + (word0 >> 2);
 #pragma unroll
-  for (int i = 0; i < Raw<BITS>::kWords / 4; ++i) {
+  for (int i = 0; i < NW / 4; ++i) {
     const uint4 v = __ldg(cw + i);
     r.w[4 * i] = v.x; r.w[4 * i + 1] = v.y; r.w[4 * i + 2] = v.z; r.w[4 * i + 3] = v.w;
   }
@@ -280,13 +282,23 @@ __device__ __forceinline__ float raw_zero(const Raw<BITS>& r, int j) {
   return bf16_bits_to_f32((z >> (16 * (j & 1))) & 0xFFFFu);
 }
 
+// One of up to four per-group constants, picked by a group index that may only be known at run time (a CTA of a
+// pair works on the half of the row its rank selects); with a compile-time index this folds to a[j].
+template <int G>
+__device__ __forceinline__ uint32_t pick_group(const uint32_t* a, int j) {
+  if constexpr (G == 1) return a[0];
+  else if constexpr (G == 2) return j ? a[1] : a[0];
+  else return (j & 2) ? ((j & 1) ? a[3] : a[2]) : ((j & 1) ? a[1] : a[0]);
+}
+
 // Keys: x^ = (code - zero) * step as FP16, one FMA per pair: (OFF + code) * step - (OFF + zero) * step
 // with OFF = 4 (2-bit) or 16 (4-bit) coming for free from the exponent bits OR-ed over the code.
 // Pairs are (i, i + 8) of each 16-code word (2-bit) or (i, i + 4) of each 8-code word (4-bit): the
 // contraction dimension is stored permuted, and the rotated query is stored with the same permutation.
-template <int BITS, int GROUP>
-__device__ __forceinline__ void dequant_keys(const Raw<BITS>& r, uint8_t* tile, int key) {
-  constexpr int group = GROUP;
+// Expands the NW words r.w[0 .. NW), which are words word0 .. word0 + NW - 1 of the token, into row `row` of the tile.
+template <int BITS, int GROUP, int NW = Raw<BITS>::kWords>
+__device__ __forceinline__ void dequant_keys(const Raw<BITS>& r, uint8_t* tile, int row, int word0 = 0) {
+  constexpr int G = kD / GROUP;
   constexpr float kOff = (BITS == 2) ? 4.f : 16.f;
   uint32_t step2[4], c2[4];
 #pragma unroll
@@ -298,40 +310,46 @@ __device__ __forceinline__ void dequant_keys(const Raw<BITS>& r, uint8_t* tile, 
   }
   if constexpr (BITS == 2) {
 #pragma unroll
-    for (int wi = 0; wi < 8; ++wi) {
-      const int j = (wi * 16) / group;
+    for (int wi = 0; wi < NW; ++wi) {
+      const int gw = word0 + wi;
+      const int j = (gw * 16) / GROUP;
+      const uint32_t st = pick_group<G>(step2, j), cc = pick_group<G>(c2, j);
       const uint32_t w = r.w[wi];
       uint32_t o[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const uint32_t sh = (i <= 4) ? (w << (8 - 2 * i)) : (w >> (2 * i - 8));
-        o[i] = hfma2_f16(and_or(sh, 0x03000300u, 0x44004400u), step2[j], c2[j]);
+        o[i] = hfma2_f16(and_or(sh, 0x03000300u, 0x44004400u), st, cc);
       }
-      *reinterpret_cast<uint4*>(tile + sw128_offset(key, 2 * wi)) = make_uint4(o[0], o[1], o[2], o[3]);
-      *reinterpret_cast<uint4*>(tile + sw128_offset(key, 2 * wi + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+      *reinterpret_cast<uint4*>(tile + sw128_offset(row, 2 * gw)) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(tile + sw128_offset(row, 2 * gw + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
     }
   } else {
 #pragma unroll
-    for (int wi = 0; wi < 16; ++wi) {
-      const int j = (wi * 8) / group;
+    for (int wi = 0; wi < NW; ++wi) {
+      const int gw = word0 + wi;
+      const int j = (gw * 8) / GROUP;
+      const uint32_t st = pick_group<G>(step2, j), cc = pick_group<G>(c2, j);
       const uint32_t w = r.w[wi];
       uint32_t o[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const uint32_t sh = (i <= 1) ? (w << (6 - 4 * i)) : (w >> (4 * i - 6));
-        o[i] = hfma2_f16(and_or(sh, 0x03C003C0u, 0x4C004C00u), step2[j], c2[j]);
+        o[i] = hfma2_f16(and_or(sh, 0x03C003C0u, 0x4C004C00u), st, cc);
       }
-      *reinterpret_cast<uint4*>(tile + sw128_offset(key, wi)) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(tile + sw128_offset(row, gw)) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
 }
 
 // Values: same reconstruction as BF16, channels in natural order (the output dimension cannot be permuted
 // because current-chunk values arrive unpermuted).  2-bit: one FMA per pair; 4-bit: exact subtract then
-// multiply (the 16 + zero offset times the step is not always representable in BF16).
-template <int BITS, int GROUP>
-__device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile, int key) {
-  constexpr int group = GROUP;
+// multiply (the 16 + zero offset times the step is not always representable in BF16).  Words as for the keys;
+// the 16-byte pieces land at piece index (token's piece index - piece0), so that a CTA of a pair keeps its 64
+// channels in one 64-column block.
+template <int BITS, int GROUP, int NW = Raw<BITS>::kWords>
+__device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile, int row, int word0 = 0, int piece0 = 0) {
+  constexpr int G = kD / GROUP;
   uint32_t step2[4], c2[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
@@ -342,8 +360,10 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
   }
   if constexpr (BITS == 2) {
 #pragma unroll
-    for (int wi = 0; wi < 8; ++wi) {
-      const int j = (wi * 16) / group;
+    for (int wi = 0; wi < NW; ++wi) {
+      const int gw = word0 + wi;
+      const int j = (gw * 16) / GROUP;
+      const uint32_t st = pick_group<G>(step2, j), cc = pick_group<G>(c2, j);
       const uint32_t w = r.w[wi];
       const uint32_t lo = w & 0x33333333u, hi = (w >> 2) & 0x33333333u;
       const uint32_t z1 = (lo & 0xFFFFu) | (hi << 16), z2 = (lo >> 16) | (hi & 0xFFFF0000u);
@@ -352,16 +372,18 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
       for (int i = 0; i < 4; ++i) {
         const uint32_t s1 = (i <= 1) ? (z1 << (5 - 4 * i)) : (z1 >> (4 * i - 5));
         const uint32_t s2 = (i <= 1) ? (z2 << (5 - 4 * i)) : (z2 >> (4 * i - 5));
-        o[i] = hfma2_bf16(and_or(s1, 0x00600060u, 0x40804080u), step2[j], c2[j]);
-        o[4 + i] = hfma2_bf16(and_or(s2, 0x00600060u, 0x40804080u), step2[j], c2[j]);
+        o[i] = hfma2_bf16(and_or(s1, 0x00600060u, 0x40804080u), st, cc);
+        o[4 + i] = hfma2_bf16(and_or(s2, 0x00600060u, 0x40804080u), st, cc);
       }
-      *reinterpret_cast<uint4*>(tile + sw128_offset(key, 2 * wi)) = make_uint4(o[0], o[1], o[2], o[3]);
-      *reinterpret_cast<uint4*>(tile + sw128_offset(key, 2 * wi + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+      *reinterpret_cast<uint4*>(tile + sw128_offset(row, 2 * gw - piece0)) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(tile + sw128_offset(row, 2 * gw + 1 - piece0)) = make_uint4(o[4], o[5], o[6], o[7]);
     }
   } else {
 #pragma unroll
-    for (int wi = 0; wi < 16; ++wi) {
-      const int j = (wi * 8) / group;
+    for (int wi = 0; wi < NW; ++wi) {
+      const int gw = word0 + wi;
+      const int j = (gw * 8) / GROUP;
+      const uint32_t st = pick_group<G>(step2, j), cc = pick_group<G>(c2, j);
       const uint32_t w = r.w[wi];
       const uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;
       const uint32_t z1 = (lo & 0xFFFFu) | (hi << 16), z2 = (lo >> 16) | (hi & 0xFFFF0000u);
@@ -370,10 +392,10 @@ __device__ __forceinline__ void dequant_values(const Raw<BITS>& r, uint8_t* tile
       for (int i = 0; i < 2; ++i) {
         const uint32_t s1 = (i == 0) ? (z1 << 3) : (z1 >> 5);
         const uint32_t s2 = (i == 0) ? (z2 << 3) : (z2 >> 5);
-        o[i] = hmul2_bf16(hsub2_bf16(and_or(s1, 0x00780078u, 0x41804180u), c2[j]), step2[j]);
-        o[2 + i] = hmul2_bf16(hsub2_bf16(and_or(s2, 0x00780078u, 0x41804180u), c2[j]), step2[j]);
+        o[i] = hmul2_bf16(hsub2_bf16(and_or(s1, 0x00780078u, 0x41804180u), cc), st);
+        o[2 + i] = hmul2_bf16(hsub2_bf16(and_or(s2, 0x00780078u, 0x41804180u), cc), st);
       }
-      *reinterpret_cast<uint4*>(tile + sw128_offset(key, wi)) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(tile + sw128_offset(row, gw - piece0)) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
 }
@@ -478,7 +500,14 @@ __global__ void __launch_bounds__(256) rotate_query_kernel(const RotParams p) {
 }
 
 
-template <int BITS, int GROUP>
+// PAIR: two CTAs of a cluster work as one (tcgen05 cta_group::2).  The pair shares the key and value tiles of one
+// (batch, head): CTA r owns query rows [256 r, 256 r + 256) of a 512-row unit and dequantizes (or loads) HALF of
+// every operand tile - 32 of the 64 keys of each score product's B operand, 64 of the 128 value channels - so the
+// dequantization work, the stores and the B-operand reads per SM halve.  The leader CTA (rank 0) issues every
+// MMA, with M = 256: 128 rows in each CTA's own TMEM.  Barriers the issuer waits on live in the leader and take
+// arrivals from both CTAs; barriers the issuer signals are committed to both CTAs at once.  No load is multicast:
+// each CTA fetches its own half.
+template <int BITS, int GROUP, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qr,
                     const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TParams p) {
@@ -490,6 +519,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   KVQ_TRACE_DECL;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;            // 0: the CTA that issues the MMAs
+  const int sched_id = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // which range of the schedule (one per pair)
+  const int n_sched = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  constexpr int kC = PAIR ? 2 : 1;                                // CTAs that arrive on the issuer's barriers
+  // barrier i of the issuing CTA, as an address an arrival (or a TMA completion) from either CTA can use
+  auto lead = [&](int i) -> uint32_t { return PAIR ? map_to_cta(cx.bar(i), 0) : cx.bar(i); };
+  auto arrive_lead = [&](int i) { if constexpr (PAIR) mbar_arrive_cluster(lead(i)); else mbar_arrive(cx.bar(i)); };
+  auto expect_tx_lead = [&](int i, uint32_t bytes) {
+    if constexpr (PAIR) mbar_arrive_expect_tx_cluster(lead(i), bytes); else mbar_arrive_expect_tx(cx.bar(i), bytes);
+  };
+  // first query row of this CTA in schedule unit `unit` (a unit is 256 rows, 512 for a pair)
+  auto unit_row0 = [&](int unit, int bh) { return (unit - bh * p.q_blocks) * (2 * kC * kBlockM) + (int)rank * 2 * kBlockM; };
   const int n_rt = (p.n_cur + kBlockN - 1) / kBlockN;
   const int n_ct = (p.n_cached + kBlockN - 1) / kBlockN;
   const int T = n_rt + n_ct;
@@ -497,26 +538,26 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (tid == 0) {
     misc[1] = 0;
-    mbar_init(cx.bar(kQFull), 1);
+    mbar_init(cx.bar(kQFull), kC);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(cx.bar(kKFull + s), 129);   // 128 dequant threads + the TMA thread, every tile
-      mbar_init(cx.bar(kVFull + s), 129);
+      mbar_init(cx.bar(kKFull + s), 129 * kC);   // 128 dequant threads + the TMA thread (of each CTA), every tile
+      mbar_init(cx.bar(kVFull + s), 129 * kC);
       mbar_init(cx.bar(kKEmpty + s), 2);    // both MMA issuers commit
       mbar_init(cx.bar(kVEmpty + s), 2);
       mbar_init(cx.bar(kSFull + s), 1);
       mbar_init(cx.bar(kSFull + 2 + s), 1);
-      mbar_init(cx.bar(kPFull + s), 128);   // the four softmax warps of a query tile
-      mbar_init(cx.bar(kPFull + 2 + s), 128);
+      mbar_init(cx.bar(kPFull + s), 128 * kC);   // the four softmax warps of a query tile (of each CTA)
+      mbar_init(cx.bar(kPFull + 2 + s), 128 * kC);
       mbar_init(cx.bar(kODone + s), 1);
       mbar_init(cx.bar(kODone + 2 + s), 1);
     }
     mbar_init(cx.bar(kQCurDone), 2);
-    mbar_init(cx.bar(kQRotFull), 129);   // 128 dequant threads (bias rows) + the TMA thread (rotated query tile)
+    mbar_init(cx.bar(kQRotFull), 129 * kC);   // 128 dequant threads (bias rows) + the TMA thread (rotated query tile)
     mbar_init(cx.bar(kDrain + 0), 1);
     mbar_init(cx.bar(kDrain + 1), 1);
     mbar_init(cx.bar(kQEmpty), 2);
-    mbar_init(cx.bar(kOFree + 0), 128);
-    mbar_init(cx.bar(kOFree + 1), 128);
+    mbar_init(cx.bar(kOFree + 0), 128 * kC);
+    mbar_init(cx.bar(kOFree + 1), 128 * kC);
     fence_barrier_init();
     prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_qr); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
   }
@@ -524,12 +565,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   for (int i = tid; i < 4 * kXBytes / 16; i += kThreads)
     reinterpret_cast<uint4*>(smem + kOffAx)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 0) {
-    tmem_alloc(sbase + kOffMisc, 512);
-    tmem_relinquish();
+    if constexpr (PAIR) { tmem_alloc_pair(sbase + kOffMisc, 512); tmem_relinquish_pair(); }
+    else { tmem_alloc(sbase + kOffMisc, 512); tmem_relinquish(); }
   }
   fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();        // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
   // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_q aliases the first 64 columns of S_q.
@@ -539,56 +581,74 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
-      Schedule sch(blockIdx.x, gridDim.x, p);
+      auto load_q = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+        if constexpr (PAIR) tma_load_4d_pair(dst, map, bar, c0, c1, c2, c3);
+        else tma_load_4d(dst, map, bar, c0, c1, c2, c3);
+      };
+      Schedule sch(sched_id, n_sched, p);
       Segment sg;
       int it = 0, nseg = 0, issued_it = -1, rot_seg = -1;
       bool ok = true;
       while (ok && sch.next(sg)) {
         const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
-        const int row0 = (sg.unit - bh * p.q_blocks) * (2 * kBlockM);
+        const int row0 = unit_row0(sg.unit, bh);
         // the query buffer is free once every score MMA of the previous segment has retired (the MMA warp says so
         // in its last iteration, before the last P V products)
         if (!(ok = cx.wait(kQEmpty, (nseg & 1) ^ 1, 100))) break;
         // a segment that starts in the cache never needs the unrotated query: load the rotated one right away
         const bool cached0 = sg.tb >= n_rt;
-        mbar_arrive_expect_tx(cx.bar(kQFull), 2 * kTileBytes);
+        expect_tx_lead(kQFull, 2 * kTileBytes);
         for (int qt = 0; qt < 2; ++qt)
           for (int kb = 0; kb < 2; ++kb)
-            tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, cached0 ? &tm_qr : &tm_q, cx.bar(kQFull), kb * 64, row0 + qt * kBlockM, h, b);
-        if (cached0 || sg.te <= n_rt) mbar_arrive(cx.bar(kQRotFull));   // this thread's share of the phase
+            load_q(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, cached0 ? &tm_qr : &tm_q, lead(kQFull), kb * 64, row0 + qt * kBlockM, h, b);
+        if (cached0 || sg.te <= n_rt) arrive_lead(kQRotFull);   // this thread's share of the phase
         for (int t = sg.tb; t < sg.te; ++t, ++it) {
           const int s = it & 1;
           const uint32_t ph = (it >> 1) & 1;
           if (t == n_rt && !cached0) {
             // first cached tile: once no MMA reads the unrotated query any more, the rotated tile replaces it
             if (!(ok = cx.wait(kQCurDone, nseg & 1, 103))) break;
-            mbar_arrive_expect_tx(cx.bar(kQRotFull), 2 * kTileBytes);
+            expect_tx_lead(kQRotFull, 2 * kTileBytes);
             for (int qt = 0; qt < 2; ++qt)
               for (int kb = 0; kb < 2; ++kb)
-                tma_load_4d(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, &tm_qr, cx.bar(kQRotFull), kb * 64, row0 + qt * kBlockM, h, b);
+                load_q(sbase + kOffQ + qt * kTileBytes + kb * kHalfTile, &tm_qr, lead(kQRotFull), kb * 64, row0 + qt * kBlockM, h, b);
             rot_seg = nseg;
           }
           if (!(ok = cx.wait(kKEmpty + s, ph ^ 1, 101))) break;
           if (t < n_rt) {
-            mbar_arrive_expect_tx(cx.bar(kKFull + s), kTileBytes);
-            for (int kb = 0; kb < 2; ++kb)
-              tma_load_4d(sbase + kOffK + s * kTileBytes + kb * kHalfTile, &tm_k, cx.bar(kKFull + s), kb * 64, t * kBlockN, h, b);
+            expect_tx_lead(kKFull + s, kTileBytes / kC);
+            if constexpr (PAIR) {
+              // this CTA's 32 keys of each half of the tile (local rows 32 hf .. 32 hf + 31): boxes of 32 rows
+              for (int hf = 0; hf < 2; ++hf)
+                for (int kb = 0; kb < 2; ++kb)
+                  tma_load_4d_pair(sbase + kOffK + s * kTileBytes + kb * kHalfTile + hf * 32 * 128, &tm_k, lead(kKFull + s), kb * 64,
+                              t * kBlockN + 64 * hf + 32 * (int)rank, h, b);
+            } else {
+              for (int kb = 0; kb < 2; ++kb)
+                tma_load_4d(sbase + kOffK + s * kTileBytes + kb * kHalfTile, &tm_k, cx.bar(kKFull + s), kb * 64, t * kBlockN, h, b);
+            }
           } else {
-            mbar_arrive(cx.bar(kKFull + s));
+            arrive_lead(kKFull + s);
           }
           if (!(ok = cx.wait(kVEmpty + s, ph ^ 1, 102))) break;
           if (t < n_rt) {
-            mbar_arrive_expect_tx(cx.bar(kVFull + s), kTileBytes);
-            for (int kb = 0; kb < 2; ++kb)
-              tma_load_4d(sbase + kOffV + s * kTileBytes + kb * kHalfTile, &tm_v, cx.bar(kVFull + s), kb * 64, t * kBlockN, h, b);
+            expect_tx_lead(kVFull + s, kTileBytes / kC);
+            if constexpr (PAIR) {   // this CTA's 64 value channels of all 128 keys: one 64-column block
+              tma_load_4d_pair(sbase + kOffV + s * kTileBytes, &tm_v, lead(kVFull + s), 64 * (int)rank, t * kBlockN, h, b);
+            } else {
+              for (int kb = 0; kb < 2; ++kb)
+                tma_load_4d(sbase + kOffV + s * kTileBytes + kb * kHalfTile, &tm_v, cx.bar(kVFull + s), kb * 64, t * kBlockN, h, b);
+            }
             issued_it = it;
           } else {
-            mbar_arrive(cx.bar(kVFull + s));
+            arrive_lead(kVFull + s);
           }
         }
         ++nseg;
       }
-      if (*cx.abort) {   // drain: give loads already in flight a bounded time to land before the CTA exits
+      // drain: give loads already in flight a bounded time to land before the CTA exits (of a pair, the barriers
+      // are the leader's and count both CTAs' bytes; the peer stays until the leader has come through, below)
+      if (*cx.abort && rank == 0) {
         if (nseg > 0) cx.drain(kQFull, (nseg - 1) & 1);
         if (rot_seg >= 0) cx.drain(kQRotFull, rot_seg & 1);
         if (issued_it >= 0) {
@@ -607,12 +667,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // of this tile: per (half, query tile) the issuer waits for that half of P, issues O += P V over its 64 keys
     // and then at once S = Q K^T of the same half of the NEXT tile into the columns P has just left.  The tensor
     // pipe executes this thread's MMAs in order, so the new scores cannot overtake the product that reads P.
-    {
+    // Of a pair only the leader CTA issues (M = 256: its own 128 rows and the peer's); the peer's two warps idle.
+    if (rank == 0) {
       const bool leader = elect_one();
       const int qt = warp - 1;
-      const uint32_t idesc_bf16 = make_idesc_bf16(128, 64, 0, 0);
+      constexpr int kM = PAIR ? 256 : 128;
+      const uint32_t idesc_bf16 = make_idesc_bf16(kM, 64, 0, 0);
       const uint32_t idesc_f16 = idesc_bf16 & ~((7u << 7) | (7u << 10));     // A, B format 0 = FP16
-      const uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);              // B (values) is MN-major
+      const uint32_t idesc_pv = make_idesc_bf16(kM, 128, 0, 1);               // B (values) is MN-major
+      // commit: one arrival when every MMA issued so far has completed; of a pair, on the barrier of both CTAs
+      auto commit = [&](int i) { if constexpr (PAIR) tc_commit_pair(cx.bar(i), (uint16_t)3); else tc_commit(cx.bar(i)); };
       // Descriptors are built once; stepping along K only adds a constant to the 14-bit address field
       // (all operand tiles live below 256 KiB of shared memory, so the field cannot overflow).
       const uint64_t dq0 = make_smem_desc(sbase + kOffQ, 16, 1024, kLayoutSw128);
@@ -625,20 +689,35 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (!leader) return;
         const uint32_t idesc = cached ? idesc_f16 : idesc_bf16;
         const uint64_t qd = dq0 + (uint64_t)(qt * (kTileBytes >> 4));
-        const uint64_t kd = dk0 + (uint64_t)(s * (kTileBytes >> 4) + hf * (64 * 128 >> 4));   // key rows are 128 bytes
+        // key rows are 128 bytes; a half is 64 rows of the stage, or each CTA's 32 of them for a pair
+        const uint64_t kd = dk0 + (uint64_t)(s * (kTileBytes >> 4) + hf * ((64 / kC) * 128 >> 4));
         const uint32_t d_tmem = tmem + qt * 128 + hf * 64;
         constexpr int kBlk = kHalfTile >> 4;
-        mma_ss_off<0>(d_tmem, qd, kd, idesc, 0);
-        mma_ss_off<2>(d_tmem, qd, kd, idesc, 1);
-        mma_ss_off<4>(d_tmem, qd, kd, idesc, 1);
-        mma_ss_off<6>(d_tmem, qd, kd, idesc, 1);
-        mma_ss_off<kBlk>(d_tmem, qd, kd, idesc, 1);
-        mma_ss_off<kBlk + 2>(d_tmem, qd, kd, idesc, 1);
-        mma_ss_off<kBlk + 4>(d_tmem, qd, kd, idesc, 1);
-        mma_ss_off<kBlk + 6>(d_tmem, qd, kd, idesc, 1);
-        if (cached && p.correction)   // rows 64 hf .. of the 128 x 16 bias tile: 8-row groups are 256 bytes apart
-          mma_ss(d_tmem, dax0 + (uint64_t)(qt * (kXBytes >> 4)), dbx0 + (uint64_t)(s * (kXBytes >> 4) + hf * (8 * 256 >> 4)), idesc_bf16, 1);
-        tc_commit(cx.bar(kSFull + 2 * hf + qt));
+        // rows 64 hf .. (32 hf .. for a pair) of the bias tile: 8-row groups are 256 bytes apart
+        const uint64_t axd = dax0 + (uint64_t)(qt * (kXBytes >> 4));
+        const uint64_t bxd = dbx0 + (uint64_t)(s * (kXBytes >> 4) + hf * ((8 / kC) * 256 >> 4));
+        if constexpr (PAIR) {
+          mma_ss_off_pair<0>(d_tmem, qd, kd, idesc, 0);
+          mma_ss_off_pair<2>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off_pair<4>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off_pair<6>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off_pair<kBlk>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off_pair<kBlk + 2>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off_pair<kBlk + 4>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off_pair<kBlk + 6>(d_tmem, qd, kd, idesc, 1);
+          if (cached && p.correction) mma_ss_pair(d_tmem, axd, bxd, idesc_bf16, 1);
+        } else {
+          mma_ss_off<0>(d_tmem, qd, kd, idesc, 0);
+          mma_ss_off<2>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off<4>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off<6>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off<kBlk>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off<kBlk + 2>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off<kBlk + 4>(d_tmem, qd, kd, idesc, 1);
+          mma_ss_off<kBlk + 6>(d_tmem, qd, kd, idesc, 1);
+          if (cached && p.correction) mma_ss(d_tmem, axd, bxd, idesc_bf16, 1);
+        }
+        commit(kSFull + 2 * hf + qt);
       };
       // O_qt += P V over keys 64 hf .. 64 hf + 63 of stage s; P (BF16 pairs) sits in the first 32 of that half's
       // score columns
@@ -646,13 +725,20 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (!leader) return;
         const uint64_t vd = dv0 + (uint64_t)(s * (kTileBytes >> 4) + hf * (4 * 128));
         const uint32_t d_tmem = tmem + 256 + qt * 128, a_tmem = tmem + qt * 128 + hf * 64;
-        mma_ts_off<0 * 128>(d_tmem, a_tmem + 0, vd, idesc_pv, accumulate ? 1u : 0u);
-        mma_ts_off<1 * 128>(d_tmem, a_tmem + 8, vd, idesc_pv, 1);
-        mma_ts_off<2 * 128>(d_tmem, a_tmem + 16, vd, idesc_pv, 1);
-        mma_ts_off<3 * 128>(d_tmem, a_tmem + 24, vd, idesc_pv, 1);
-        tc_commit(cx.bar(kODone + 2 * hf + qt));
+        if constexpr (PAIR) {
+          mma_ts_off_pair<0 * 128>(d_tmem, a_tmem + 0, vd, idesc_pv, accumulate ? 1u : 0u);
+          mma_ts_off_pair<1 * 128>(d_tmem, a_tmem + 8, vd, idesc_pv, 1);
+          mma_ts_off_pair<2 * 128>(d_tmem, a_tmem + 16, vd, idesc_pv, 1);
+          mma_ts_off_pair<3 * 128>(d_tmem, a_tmem + 24, vd, idesc_pv, 1);
+        } else {
+          mma_ts_off<0 * 128>(d_tmem, a_tmem + 0, vd, idesc_pv, accumulate ? 1u : 0u);
+          mma_ts_off<1 * 128>(d_tmem, a_tmem + 8, vd, idesc_pv, 1);
+          mma_ts_off<2 * 128>(d_tmem, a_tmem + 16, vd, idesc_pv, 1);
+          mma_ts_off<3 * 128>(d_tmem, a_tmem + 24, vd, idesc_pv, 1);
+        }
+        commit(kODone + 2 * hf + qt);
       };
-      Schedule sch(blockIdx.x, gridDim.x, p);
+      Schedule sch(sched_id, n_sched, p);
       Segment sg;
       int it = 0, nseg = 0;
       bool ok = true;
@@ -674,10 +760,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const bool has_pv = t >= sg.tb, has_qk = t + 1 < sg.te, first = t == sg.tb;
           const bool rot = has_qk && t + 1 == t_rot;
           KVQ_STAMP(32);
-          if (rot && !has_pv && leader) tc_commit(cx.bar(kQCurDone));      // the segment starts in the cache
+          if (rot && !has_pv && leader) commit(kQCurDone);      // the segment starts in the cache
           // last iteration: every score MMA of the segment is issued, so the query buffer (and the bias rows) can
           // be handed to the next segment while the last P V products still run
-          if (!has_qk && leader) tc_commit(cx.bar(kQEmpty));
+          if (!has_qk && leader) commit(kQEmpty);
           const int n_ops = rot ? 4 : 2;
 #pragma unroll 1
           for (int op = 0; op < n_ops; ++op) {
@@ -690,7 +776,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               KVQ_STAMP(34);
               tc_fence_after();
               issue_pv(s, hf, !(first && hf == 0));
-              if (op == 1 && leader) tc_commit(cx.bar(kVEmpty + s));
+              if (op == 1 && leader) commit(kVEmpty + s);
               KVQ_STAMP(10 + qt);
             }
             if (has_qk && (!rot || op >= 2)) {
@@ -702,8 +788,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
               KVQ_STAMP(36);
               issue_qk(s1, hf, t + 1 >= n_rt);
               if (hf == 1 && leader) {
-                tc_commit(cx.bar(kKEmpty + s1));
-                if (t + 1 == t_lastcur) tc_commit(cx.bar(kQCurDone));
+                commit(kKEmpty + s1);
+                if (t + 1 == t_lastcur) commit(kQCurDone);
               }
               KVQ_STAMP(14 + qt);
             }
@@ -713,7 +799,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         ++nseg;
       }
       // everything issued so far must have retired before TMEM is freed
-      if (leader) tc_commit(cx.bar(kDrain + qt));
+      if (leader) commit(kDrain + qt);
       cx.drain(kDrain + qt, 0);
     }
   }
@@ -732,7 +818,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t s_addr = tmem + lane_addr + qt * 128;      // scores of half hf at columns 64 hf; P over their first 32
     const uint32_t o_addr = tmem + lane_addr + 256 + qt * 128;
     const float c_row = p.scale_log2;
-    Schedule sch(blockIdx.x, gridDim.x, p);
+    Schedule sch(sched_id, n_sched, p);
     Segment sg;
     int it = 0, nseg = 0;
     bool ok = true;
@@ -801,7 +887,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (cached) lcac += sum2.x + sum2.y; else lcur += sum2.x + sum2.y;
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(cx.bar(kPFull + 2 * hf + qt));
+          arrive_lead(kPFull + 2 * hf + qt);
           KVQ_STAMP(4 + hf);
           fresh = false;
         }
@@ -814,7 +900,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       ok = __all_sync(0xFFFFFFFFu, cx.wait(kODone + 2 + qt, (it - 1) & 1, 303));            // the last product of the segment is a second half
       if (!ok) break;
       tc_fence_after();
-      const int row = (sg.unit - bh * p.q_blocks) * (2 * kBlockM) + r256;
+      const int row = unit_row0(sg.unit, bh) + r256;
       // a whole unit writes its rows of the output; a partial segment writes the same normalised rows into its
       // slot, with the statistics the merge kernel weighs them by
       const float l = lcur + lcac;
@@ -832,7 +918,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tmem_wait_ld();
         if (hf == 1) {                               // the whole row is in registers: O can be overwritten
           tc_fence_before();
-          mbar_arrive(cx.bar(kOFree + qt));
+          arrive_lead(kOFree + qt);
         }
         if (store) {
 #pragma unroll
@@ -863,7 +949,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // ================= dequant warps =================
     setmaxnreg_dec<kRegsDequant>();
     const int dt = tid - 12 * 32;          // 0..127: the key of the tile this thread expands
-    Schedule sch(blockIdx.x, gridDim.x, p);
+    // One CTA: thread dt expands key dt of the tile, keys and values.  A CTA of a pair expands half of each
+    // tile: of the keys, its 32 keys of either half tile (local row dt / 2 = 32 hf + j is key 64 hf + 32 rank + j),
+    // two threads per key with 64 channels each; of the values, channels [64 rank, 64 rank + 64) of key dt.
+    constexpr int kNW = Raw<BITS>::kWords / kC;                    // code words per thread and tile (keys or values)
+    const int k_row = PAIR ? (dt >> 1) : dt;                       // row of the key stage this thread writes
+    const int k_key = PAIR ? 64 * (k_row >> 5) + 32 * (int)rank + (k_row & 31) : dt;   // its key within the tile
+    const int k_word0 = PAIR ? (dt & 1) * kNW : 0;                 // first code word of the key it expands
+    const int v_word0 = PAIR ? (int)rank * kNW : 0;                // first code word of value row dt it expands
+    const int v_piece0 = PAIR ? (int)rank * 8 : 0;                 // its 16-byte pieces start at piece 0 of the block
+    Schedule sch(sched_id, n_sched, p);
     Segment sg;
     int it = 0, nseg = 0;
     bool ok = true;
@@ -879,37 +974,40 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       };
       const int t_rot = max(sg.tb, n_rt);          // first cached tile of the segment: the query is rotated there
       if (sg.te > n_rt) {
-        const int k0 = (t_rot - n_rt) * kBlockN + dt;
-        load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k0), k0 < p.n_cached);
-        load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(k0), k0 < p.n_cached);
+        const int k0 = (t_rot - n_rt) * kBlockN + k_key, v0 = (t_rot - n_rt) * kBlockN + dt;
+        load_raw<BITS, G, kNW>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k0), k0 < p.n_cached, k_word0);
+        load_raw<BITS, G, kNW>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(v0), v0 < p.n_cached, v_word0);
       }
       for (int t = sg.tb; t < sg.te; ++t, ++it) {
         const int s = it & 1;
         const uint32_t ph = (it >> 1) & 1;
         const int ct = t - n_rt;
-        const int k1 = (ct + 1) * kBlockN + dt;    // this thread's key in the next tile
+        const int k1 = (ct + 1) * kBlockN + k_key, v1 = (ct + 1) * kBlockN + dt;   // this thread's keys in the next tile
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kKEmpty + s, ph ^ 1, 401));
         if (!ok) break;
         KVQ_STAMP(22);
         if (ct >= 0) {
-          dequant_keys<BITS, GROUP>(rk, smem + kOffK + s * kTileBytes, dt);
-          if (p.correction) {   // B_extra row: step_j^2, exact in BF16
+          dequant_keys<BITS, GROUP, kNW>(rk, smem + kOffK + s * kTileBytes, k_row, k_word0);
+          if (p.correction && k_word0 == 0) {   // B_extra row: step_j^2, exact in BF16
             const float d0 = raw_step<BITS>(rk, 0), d1 = raw_step<BITS>(rk, 1), d2 = raw_step<BITS>(rk, 2), d3 = raw_step<BITS>(rk, 3);
             const uint32_t b01 = pack_bf16x2(d0 * d0, G > 1 ? d1 * d1 : 0.f), b23 = pack_bf16x2(G > 2 ? d2 * d2 : 0.f, G > 3 ? d3 * d3 : 0.f);
             // columns 0..3 meet the high parts of A_extra, columns 4..7 the low parts
-            *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(dt, 0)) = make_uint4(b01, b23, b01, b23);
+            *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(k_row, 0)) = make_uint4(b01, b23, b01, b23);
           }
           fence_proxy_async_smem();
-          if (t + 1 < sg.te) load_raw<BITS, G>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k1), k1 < p.n_cached);
+          if (t + 1 < sg.te) load_raw<BITS, G, kNW>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k1), k1 < p.n_cached, k_word0);
         }
-        mbar_arrive(cx.bar(kKFull + s));
+        arrive_lead(kKFull + s);
         KVQ_STAMP(20);
         if (t == t_rot) {
           // ---- A_extra: -(sigma/24) nu rows of this unit's 256 queries, written by the pre-pass ----
           // (the new query tile being in means every MMA of the previous segment, which read the old rows, retired)
-          ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, nseg & 1, 402));
+          // (of a pair that barrier is the leader's alone; both CTAs see "query buffer free", which the issuer commits
+          // once the previous segment's score MMAs, the readers of the old rows, are all issued and retired)
+          if constexpr (PAIR) ok = __all_sync(0xFFFFFFFFu, cx.wait(kQEmpty, (nseg & 1) ^ 1, 402));
+          else ok = __all_sync(0xFFFFFFFFu, cx.wait(kQFull, nseg & 1, 402));
           if (!ok) break;
-          const int row0 = (sg.unit - bh * p.q_blocks) * (2 * kBlockM);
+          const int row0 = unit_row0(sg.unit, bh);
 #pragma unroll
           for (int qt = 0; qt < 2; ++qt) {
             const int row = row0 + qt * kBlockM + dt;
@@ -918,29 +1016,32 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             *reinterpret_cast<uint4*>(smem + kOffAx + qt * kXBytes + xtile_offset(dt, 0)) = a;
           }
           fence_proxy_async_smem();
-          mbar_arrive(cx.bar(kQRotFull));
+          arrive_lead(kQRotFull);
         }
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kVEmpty + s, ph ^ 1, 404));
         if (!ok) break;
         KVQ_STAMP(23);
         if (ct >= 0) {
-          dequant_values<BITS, GROUP>(rv, smem + kOffV + s * kTileBytes, dt);
+          dequant_values<BITS, GROUP, kNW>(rv, smem + kOffV + s * kTileBytes, dt, v_word0, v_piece0);
           fence_proxy_async_smem();
-          if (t + 1 < sg.te) load_raw<BITS, G>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(k1), k1 < p.n_cached);
+          if (t + 1 < sg.te) load_raw<BITS, G, kNW>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(v1), v1 < p.n_cached, v_word0);
         }
-        mbar_arrive(cx.bar(kVFull + s));
+        arrive_lead(kVFull + s);
         KVQ_STAMP(21);
       }
       if (!ok) break;
-      if (sg.te <= n_rt) mbar_arrive(cx.bar(kQRotFull));   // no rotation in this segment: keep the phase count in step
+      if (sg.te <= n_rt) arrive_lead(kQRotFull);   // no rotation in this segment: keep the phase count in step
       ++nseg;
     }
   }
 
   __syncthreads();
+  // A pair leaves together: neither CTA's shared memory or TMEM may go while the other still arrives on its
+  // barriers or the leader's MMAs still read its operands (every role above has come out through bounded waits).
+  if constexpr (PAIR) cluster_sync_all();
   if (warp == 0) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    if constexpr (PAIR) tmem_dealloc_pair(tmem, 512); else tmem_dealloc(tmem, 512);
     // a wait that gave up left its diagnostic code in the abort word: report the first one
     if (lane == 0 && misc[1] != 0 && p.status) atomicCAS(p.status, 0, misc[1]);
   }
@@ -948,8 +1049,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
 // Combines the partial results of every unit whose key tiles were split over several CTAs.
 // grid (n_units - n_whole, 16): a block handles 16 rows x 128 columns; thread = (8-column piece, row).
-__global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_ctas) {
-  const int unit = p.n_whole + blockIdx.x;
+// pair = 1: the schedule's units are 512 rows worked on by CTA pairs (n_ctas counts pairs); the grid has two blocks
+// per unit in x, one for each 256-row half, whose partial results are those of the CTAs of that rank.
+__global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_ctas, int pair) {
+  const int su = pair ? blockIdx.x >> 1 : blockIdx.x, rank = pair ? blockIdx.x & 1 : 0, kc = pair ? 2 : 1;
+  const int unit = p.n_whole + su;
   const int T = p.tiles;
   // Which CTAs worked on this unit, found once per block (64-bit divisions): CTA c owns the tile steps
   // [W c / n_ctas, W (c + 1) / n_ctas) of the split part.  A CTA's slot 0 belongs to the unit its range starts
@@ -957,7 +1061,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
   __shared__ int s_first, s_last, s_first_slot;
   if (threadIdx.x == 0) {
     const long long W = (long long)(p.n_units - p.n_whole) * T;     // tile steps of the split part
-    const long long g_lo = (long long)blockIdx.x * T, g_hi = g_lo + T;
+    const long long g_lo = (long long)su * T, g_hi = g_lo + T;
     // floor(W c / n) <= g  <=>  W c < (g + 1) n: the exact tests need no division, a double gives the first guess
     auto starts_by = [&](long long c, long long g) { return W * c < (g + 1) * n_ctas; };
     auto owner = [&](long long g) {
@@ -981,11 +1085,12 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const TParams p, int n_
   const int cg = threadIdx.x >> 4, rr = threadIdx.x & 15;
   const int bh = unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
   const int r256 = blockIdx.y * 16 + rr;
-  const int row = (unit - bh * p.q_blocks) * 256 + r256;
+  const int row = (unit - bh * p.q_blocks) * (256 * kc) + rank * 256 + r256;
   if (row - rr >= p.m_tokens) return;                  // the same for the whole block: no rows left in this block
   // Partials are taken four at a time with all of their loads issued before any is used: a thread moves only
   // 16 bytes per partial, so the kernel lives on loads in flight.
-  auto slot_of = [&](int c) { return p.partial + (size_t)(2 * c + (c == c_first ? first_slot : 0)) * kSlotBytes; };
+  // CTA c of the schedule is CTA kc * c + rank of the grid; every CTA of the grid has two slots
+  auto slot_of = [&](int c) { return p.partial + (size_t)(2 * (kc * c + rank) + (c == c_first ? first_slot : 0)) * kSlotBytes; };
   float m = -INFINITY;
   for (int c0 = c_first; c0 <= c_last; c0 += 4) {
     float mm[4];
@@ -1076,11 +1181,12 @@ bool map_strides(kvq_strides s, int64_t tokens, int heads, int batch, cuuint64_t
 }
 
 // [batch, heads, tokens, 128] BF16 tensor -> 4-D map with a 64-column x 128-row box, 128-byte swizzle.
-int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, kvq_strides s, int64_t tokens, int heads, int batch) {
+int make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, kvq_strides s, int64_t tokens, int heads, int batch,
+             int box_rows = kBlockN) {
   cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)batch};
   cuuint64_t strides[3];
   if (!map_strides(s, tokens, heads, batch, strides)) return KVQ_ERR_UNSUPPORTED;
-  cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 1, 1};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1105,8 +1211,8 @@ int num_sms() {
 //    tile steps per CTA (a second prologue and epilogue, FP32 partial results, the merge kernel): split
 //    when the idle time is worth more than that.
 struct Plan { int ctas; int n_whole; };
-Plan plan_grid(int64_t n_units, int64_t tiles) {
-  const int sms = num_sms();
+Plan plan_grid(int64_t n_units, int64_t tiles, bool pair = false) {
+  const int sms = pair ? num_sms() / 2 : num_sms();      // CTAs, or CTA pairs, that run at once
   if (n_units >= sms) {
     const int64_t r = n_units % sms;
     return {sms, (int)((r == 0 || 2 * r > sms) ? n_units : n_units - r)};
@@ -1120,24 +1226,34 @@ Plan plan_grid(int64_t n_units, int64_t tiles) {
   return {(int)(c < 1 ? 1 : c), 0};
 }
 
-template <int BITS, int GROUP>
+template <int BITS, int GROUP, bool PAIR>
 int launch(const CUtensorMap& mq, const CUtensorMap& mqr, const CUtensorMap& mk, const CUtensorMap& mv, const TParams& p,
            const RotParams& rp, dim3 grid, cudaStream_t st) {
   static PerDevice configured;                       // the attribute is per device
   int dev = 0;
   { const int r = current_device(&dev); if (r != KVQ_OK) return r; }
   if (configured.first(dev)) {
-    KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_tcgen05_kernel<BITS, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    KVQ_CUDA_TRY(cudaFuncSetAttribute(attn_tcgen05_kernel<BITS, GROUP, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured.done(dev);
   }
   if (rp.qr) {                      // there are cached keys: rotate the query chunk first
     rotate_query_kernel<BITS, GROUP><<<dim3((unsigned)((rp.m_tokens + 15) / 16), (unsigned)(p.n_units / p.q_blocks)), 256, 0, st>>>(rp);
     KVQ_CUDA_TRY(cudaGetLastError());
   }
-  attn_tcgen05_kernel<BITS, GROUP><<<grid, kThreads, kSmemBytes, st>>>(mq, mqr, mk, mv, p);
+  if constexpr (PAIR) {             // grid.x counts pairs: two CTAs each, launched as clusters of two
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * grid.x); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    KVQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tcgen05_kernel<BITS, GROUP, true>, mq, mqr, mk, mv, p));
+  } else {
+    attn_tcgen05_kernel<BITS, GROUP, false><<<grid, kThreads, kSmemBytes, st>>>(mq, mqr, mk, mv, p);
+  }
   KVQ_CUDA_TRY(cudaGetLastError());
   if (p.n_whole != p.n_units) {   // units were split over CTAs: combine their partial results
-    attn_merge_kernel<<<dim3((unsigned)(p.n_units - p.n_whole), 16), 256, 0, st>>>(p, (int)grid.x);
+    attn_merge_kernel<<<dim3((unsigned)((p.n_units - p.n_whole) * (PAIR ? 2 : 1)), 16), 256, 0, st>>>(p, (int)grid.x, PAIR ? 1 : 0);
     KVQ_CUDA_TRY(cudaGetLastError());
   }
   return KVQ_OK;
@@ -1157,8 +1273,9 @@ bool attn_tcgen05_addressable(const AttnArgs& a) {
 }
 
 static void schedule_shape(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur,
-                           int64_t* q_blocks, int64_t* n_units, int64_t* tiles) {
-  *q_blocks = (m_tokens + 2 * kBlockM - 1) / (2 * kBlockM);
+                           int64_t* q_blocks, int64_t* n_units, int64_t* tiles, bool pair = false) {
+  const int64_t rows = (pair ? 4 : 2) * kBlockM;           // query rows of a unit: two tiles per CTA
+  *q_blocks = (m_tokens + rows - 1) / rows;
   *n_units = (int64_t)d->batch * d->heads * *q_blocks;
   *tiles = (n_cur + kBlockN - 1) / kBlockN + (cache_len + kBlockN - 1) / kBlockN;
 }
@@ -1171,20 +1288,20 @@ static size_t rot_area_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t
   return (rows * (2 * kD + 16) + 255) / 256 * 256;
 }
 
-size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur) {
+size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur, bool pair) {
   if (m_tokens <= 0) return 0;
   int64_t qb, nu, tiles;
-  schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
-  const Plan pl = plan_grid(nu, tiles);
-  const size_t slots = pl.n_whole != nu ? (size_t)pl.ctas * 2 * kSlotBytes : 0;
+  schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles, pair);
+  const Plan pl = plan_grid(nu, tiles, pair);
+  const size_t slots = pl.n_whole != nu ? (size_t)pl.ctas * (pair ? 2 : 1) * 2 * kSlotBytes : 0;
   return rot_area_bytes(d, cache_len, m_tokens) + slots;
 }
 
-int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur) {
+int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur, bool pair) {
   if (m_tokens <= 0) return 0;
   int64_t qb, nu, tiles;
-  schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles);
-  const Plan pl = plan_grid(nu, tiles);
+  schedule_shape(d, cache_len, m_tokens, n_cur, &qb, &nu, &tiles, pair);
+  const Plan pl = plan_grid(nu, tiles, pair);
   return 1 + (cache_len > 0 ? 1 : 0) + (pl.n_whole != nu ? 1 : 0);   // attention, query pre-pass, merge
 }
 
@@ -1193,14 +1310,16 @@ void set_attn_wait_budget(uint32_t cycles) { g_wait_budget.store(cycles, std::me
 
 // Common tail of both entry points.  `rot_area` (rot_area_bytes() bytes, 256-byte aligned; null only when
 // there are no cached keys) receives the rotated queries; `slots` holds the partial results of split units.
-static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, uint8_t* slots) {
+static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t nu, int64_t tiles, uint8_t* rot_area, uint8_t* slots,
+                          bool pair = false) {
   const kvq_cache_desc* d = a.desc;
   EncodeTiledFn enc;
   int r = get_encode_fn(&enc);
   if (r != KVQ_OK) return r;
   CUtensorMap mq, mqr, mk, mv;
   if ((r = make_map(enc, &mq, a.q, a.qs, a.m_tokens, d->heads, d->batch)) != KVQ_OK) return r;
-  if ((r = make_map(enc, &mk, a.k_cur, a.kvs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
+  // a CTA of a pair loads its 32 keys of each half tile: boxes of 32 rows
+  if ((r = make_map(enc, &mk, a.k_cur, a.kvs, a.n_cur, d->heads, d->batch, pair ? 32 : kBlockN)) != KVQ_OK) return r;
   if ((r = make_map(enc, &mv, a.v_cur, a.vs, a.n_cur, d->heads, d->batch)) != KVQ_OK) return r;
   if ((int64_t)d->batch * d->heads > 65535) return KVQ_ERR_UNSUPPORTED;   // second grid dimension of the pre-pass
   RotParams rp{};
@@ -1235,25 +1354,29 @@ static int launch_planned(const AttnArgs& a, const Plan& pl, int64_t qb, int64_t
   p.ax_rows = rp.ax;
   p.n_whole = pl.n_whole;
   dim3 grid((unsigned)pl.ctas);
+#define KVQ_LAUNCH(B_, G_) (pair ? launch<B_, G_, true>(mq, mqr, mk, mv, p, rp, grid, a.stream) \
+                                 : launch<B_, G_, false>(mq, mqr, mk, mv, p, rp, grid, a.stream))
   if (d->bits == 2) {
-    if (d->group == 32) return launch<2, 32>(mq, mqr, mk, mv, p, rp, grid, a.stream);
-    if (d->group == 64) return launch<2, 64>(mq, mqr, mk, mv, p, rp, grid, a.stream);
-    return launch<2, 128>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+    if (d->group == 32) return KVQ_LAUNCH(2, 32);
+    if (d->group == 64) return KVQ_LAUNCH(2, 64);
+    return KVQ_LAUNCH(2, 128);
   }
-  if (d->group == 32) return launch<4, 32>(mq, mqr, mk, mv, p, rp, grid, a.stream);
-  if (d->group == 64) return launch<4, 64>(mq, mqr, mk, mv, p, rp, grid, a.stream);
-  return launch<4, 128>(mq, mqr, mk, mv, p, rp, grid, a.stream);
+  if (d->group == 32) return KVQ_LAUNCH(4, 32);
+  if (d->group == 64) return KVQ_LAUNCH(4, 64);
+  return KVQ_LAUNCH(4, 128);
+#undef KVQ_LAUNCH
 }
 
 int launch_attn_tcgen05(const AttnArgs& a) {
+  const bool pair = (a.flags & KVQ_KERNEL_MASK) == KVQ_KERNEL_TCGEN05_PAIR;
   int64_t qb, nu, tiles;
-  schedule_shape(a.desc, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles);
+  schedule_shape(a.desc, a.cache_len, a.m_tokens, a.n_cur, &qb, &nu, &tiles, pair);
   if (nu * tiles > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
-  const Plan pl = plan_grid(nu, tiles);
+  const Plan pl = plan_grid(nu, tiles, pair);
   // workspace: [rotated-query area][partial-result slots]; its size was checked by the caller
   const size_t rot = rot_area_bytes(a.desc, a.cache_len, a.m_tokens);
   uint8_t* ws = static_cast<uint8_t*>(a.workspace);
-  return launch_planned(a, pl, qb, nu, tiles, rot ? ws : nullptr, ws + rot);
+  return launch_planned(a, pl, qb, nu, tiles, rot ? ws : nullptr, ws + rot, pair);
 }
 
 

@@ -76,7 +76,7 @@ static int check_attn_args(const kvq_cache_desc* d, int64_t cache_begin, int64_t
   if (((d->flags & KVQ_RING) ? cache_len : cache_begin + cache_len) > d->capacity) return KVQ_ERR_CAPACITY;
   if (m_tokens > 0x7FFFFFFFLL || n_cur > 0x7FFFFFFFLL || cache_len > 0x7FFFFFFFLL) return KVQ_ERR_UNSUPPORTED;
   const uint32_t kern = flags & KVQ_KERNEL_MASK;
-  if (kern != KVQ_KERNEL_AUTO && kern != KVQ_KERNEL_MMA_SYNC && kern != KVQ_KERNEL_TCGEN05)
+  if (kern != KVQ_KERNEL_AUTO && kern != KVQ_KERNEL_MMA_SYNC && kern != KVQ_KERNEL_TCGEN05 && kern != KVQ_KERNEL_TCGEN05_PAIR)
     return KVQ_ERR_INVALID_ARG;
   if (flags & ~(KVQ_CORRECTION_ON | KVQ_CORRECTION_EXACT | KVQ_KERNEL_MASK)) return KVQ_ERR_INVALID_ARG;
   if ((flags & KVQ_CORRECTION_ON) && (flags & KVQ_CORRECTION_EXACT)) return KVQ_ERR_INVALID_ARG;   // one form or the other
@@ -97,9 +97,10 @@ static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur
   if (kern == KVQ_KERNEL_MMA_SYNC) return false;
   // the exact correction (a table look-up per score and group) exists in the warp-level kernel only
   const bool ok = attn_tcgen05_supports(d, m_tokens, n_cur) && !(flags & KVQ_CORRECTION_EXACT) && !(d->flags & KVQ_K_PER_CHANNEL);
-  if (kern == KVQ_KERNEL_TCGEN05 && !ok) *err = KVQ_ERR_UNSUPPORTED;
+  if ((kern == KVQ_KERNEL_TCGEN05 || kern == KVQ_KERNEL_TCGEN05_PAIR) && !ok) *err = KVQ_ERR_UNSUPPORTED;
   return ok;
 }
+static bool is_pair(uint32_t flags) { return (flags & KVQ_KERNEL_MASK) == KVQ_KERNEL_TCGEN05_PAIR; }
 
 // Checks shared by the two attention entry points, then the argument block the launchers take.
 static int check_attn_call(const kvq_cache_desc* d, int64_t cache_begin, int64_t cache_len, const void* q,
@@ -197,7 +198,7 @@ int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0);
+  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags)) : 0);
   return KVQ_OK;
 }
 
@@ -209,7 +210,7 @@ int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur) : (m_tokens > 0 ? 1 : 0)) +
+  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur, is_pair(flags)) : (m_tokens > 0 ? 1 : 0)) +
                (rotv_bytes(desc, cache_len, m_tokens, n_cur) ? 2 : 0);      // value pre-pass and output post-pass
   return KVQ_OK;
 }
@@ -232,12 +233,12 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   // Tensors TMA cannot address (a stride of 0, as in a chunk expanded over heads) go to the warp-level kernel,
   // which takes any stride; a forced tcgen05 kernel fails here, before anything is launched.
   if (tc && m_tokens > 0 && !attn_tcgen05_addressable(a)) {
-    if ((flags & KVQ_KERNEL_MASK) == KVQ_KERNEL_TCGEN05) return KVQ_ERR_UNSUPPORTED;
+    if ((flags & KVQ_KERNEL_MASK) != KVQ_KERNEL_AUTO) return KVQ_ERR_UNSUPPORTED;
     tc = false;
   }
   const size_t rotv = rotv_bytes(desc, cache_len, m_tokens, n_cur);
   {
-    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur) : 0);
+    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags)) : 0);
     if (need > 0) {
       if (!workspace || workspace_bytes < need) return KVQ_ERR_WORKSPACE;
       if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return KVQ_ERR_ALIGNMENT;

@@ -75,8 +75,9 @@ int launch_rotate_rows(const kvq_cache_desc* d, const void* src, kvq_strides ss,
 bool attn_tcgen05_supports(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur);
 // Can TMA address the call's Q, K_cur, V_cur (no zero stride in a real dimension, byte strides below 2^40)?
 bool attn_tcgen05_addressable(const AttnArgs& a);
-size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
-int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur);
+// pair: the CTA-pair form of the kernel (KVQ_KERNEL_TCGEN05_PAIR), which plans 512-row units over SM pairs
+size_t attn_tcgen05_workspace_bytes(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur, bool pair);
+int attn_tcgen05_kernel_launches(const kvq_cache_desc* d, int64_t cache_len, int64_t m_tokens, int64_t n_cur, bool pair);
 int launch_attn_tcgen05(const AttnArgs& a);
 // Cycle budget of the tcgen05 kernel's device-side waits for later launches (0 = the default of about a second).
 void set_attn_wait_budget(uint32_t cycles);

@@ -20,10 +20,12 @@ def B():
 
 
 def kernels(B, head_dim=128):
-    """Every kernel that covers the shape: the warp-level one always, the tcgen05 one for head_dim 128."""
+    """Every kernel that covers the shape: the warp-level one always, the tcgen05 ones (one CTA per 256 query
+    rows; a pair of CTAs per 512) for head_dim 128."""
     ks = [("mma_sync", B.KVQ_KERNEL_MMA_SYNC)]
     if head_dim == 128:
         ks.append(("tcgen05", B.KVQ_KERNEL_TCGEN05))
+        ks.append(("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR))
     return ks
 
 
@@ -228,32 +230,36 @@ def test_large_configs_every_head(B, name):
         rows = inputs.sample_rows(w.chunk, 128, 8, seed=w.cfg_id)
         sigma = T.sigma_of(w.head_dim)
         qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)
-        lse = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
-        mass = torch.zeros_like(lse)
-        status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        out = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05, cache_len=n,
-                                   lse=lse, cached_mass=mass, status_word=status)
-        torch.cuda.synchronize()
-        assert int(status.item()) == 0
-        got, lse_h, mass_h = T.from_dev_bf16(out), lse.cpu().numpy().astype(np.float64), mass.cpu().numpy().astype(np.float64)
+        got_by_kernel = {}
+        for kname, kflag in (("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR)):
+            lse = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
+            mass = torch.zeros_like(lse)
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            out = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_ON | kflag, cache_len=n,
+                                       lse=lse, cached_mass=mass, status_word=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0, kname
+            got_by_kernel[kname] = (T.from_dev_bf16(out), lse.cpu().numpy().astype(np.float64),
+                                    mass.cpu().numpy().astype(np.float64))
         want = list(pool.map(lambda i: O.attn_corrected(caches[i], 0, n, one(q, heads[i]), one(kc, heads[i]),
                                                          one(vc, heads[i]), sigma, correction=True, rows=rows),
                              range(len(heads))))
-    worst = (0.0, 0.0)
-    for (b, h), wnt in zip(heads, want):
-        rel, mx = T.assert_attn_close(got[b, h][rows], wnt["out"][0], f"{name} head ({b},{h})")
-        worst = (max(worst[0], rel), max(worst[1], mx))
-        assert np.abs(lse_h[b, h][rows] - wnt["lse"][0]).max() < 2e-2, (b, h)
-        assert np.abs(mass_h[b, h][rows] - wnt["cached_mass"][0]).max() < 1e-2, (b, h)
-    print(f"{name}: worst rel-L2 {worst[0]:.2e}, worst max-abs {worst[1]:.2e} over {len(heads)} heads x {len(rows)} rows")
-    # the correction-off kernel on two heads
-    out_off = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_OFF | B.KVQ_KERNEL_TCGEN05, cache_len=n)
-    got_off = T.from_dev_bf16(out_off)
+    for kname, (got, lse_h, mass_h) in got_by_kernel.items():
+        worst = (0.0, 0.0)
+        for (b, h), wnt in zip(heads, want):
+            rel, mx = T.assert_attn_close(got[b, h][rows], wnt["out"][0], f"{name} {kname} head ({b},{h})")
+            worst = (max(worst[0], rel), max(worst[1], mx))
+            assert np.abs(lse_h[b, h][rows] - wnt["lse"][0]).max() < 2e-2, (kname, b, h)
+            assert np.abs(mass_h[b, h][rows] - wnt["cached_mass"][0]).max() < 1e-2, (kname, b, h)
+        print(f"{name} {kname}: worst rel-L2 {worst[0]:.2e}, worst max-abs {worst[1]:.2e} over {len(heads)} heads x {len(rows)} rows")
+    # the correction-off kernels on two heads
     for i in (0, len(heads) - 1):
         b, h = heads[i]
         wnt = O.attn_corrected(caches[i], 0, n, one(q, heads[i]), one(kc, heads[i]), one(vc, heads[i]), sigma,
                                correction=False, rows=rows)
-        T.assert_attn_close(got_off[b, h][rows], wnt["out"][0], f"{name} head ({b},{h}) uncorrected")
+        for kname, kflag in (("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR)):
+            out_off = B.kvq_attn_corrected(g, qd, kd, vd, sigma, B.KVQ_CORRECTION_OFF | kflag, cache_len=n)
+            T.assert_attn_close(T.from_dev_bf16(out_off)[b, h][rows], wnt["out"][0], f"{name} {kname} head ({b},{h}) uncorrected")
 
 
 def test_pipeline_config_steps(B):
@@ -271,7 +277,7 @@ def test_pipeline_config_steps(B):
         q, k, v = inputs.make_chunk(w, step, need_q=check)
         if check:
             _compare(B, g, o, n, q, k, v, T.sigma_of(w.head_dim), sel, rows=rows,
-                     flags_list=None if step < 15 else [("tcgen05", B.KVQ_KERNEL_TCGEN05)])
+                     flags_list=None if step < 15 else [("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR)])
         if step < 15:
             B.kvq_quantize_append(g, T.to_dev(k), T.to_dev(v))
             n = O.quantize_append(o, n, sel(k), sel(v))

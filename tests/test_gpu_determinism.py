@@ -21,8 +21,9 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("kernel", ["KVQ_KERNEL_TCGEN05", "KVQ_KERNEL_TCGEN05_PAIR"])
 @pytest.mark.parametrize("name,heads,tokens,chunks,launches", CASES, ids=[c[0] for c in CASES])
-def test_repeated_launches_give_identical_bytes(name, heads, tokens, chunks, launches):
+def test_repeated_launches_give_identical_bytes(name, heads, tokens, chunks, launches, kernel):
     from paper_2605_26266_b200 import binding as B
     w = inputs.WORKLOADS[name]
     sigma = 1.0 / math.sqrt(w.head_dim)
@@ -39,7 +40,7 @@ def test_repeated_launches_give_identical_bytes(name, heads, tokens, chunks, lau
     for i in range(launches):
         out = torch.empty_like(q)
         lse = torch.empty(q.shape[:3], dtype=torch.float32, device="cuda")
-        B.kvq_attn_corrected(cache, q, k, v, sigma, B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05, cache_len=n,
+        B.kvq_attn_corrected(cache, q, k, v, sigma, B.KVQ_CORRECTION_ON | getattr(B, kernel), cache_len=n,
                              out=out, lse=lse, status_word=status)
         B.kvq_quantize_append(cache, k, v, cache_len=n)          # the append of the step, every time at the same place
         if ref_out is None:

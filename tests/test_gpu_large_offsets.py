@@ -46,7 +46,7 @@ def test_append_and_attention_at_the_end_of_a_multi_gigabyte_cache():
 
     q, kr, vr = inputs.make_chunk(w, 1, tokens=m)
     want = O.attn_corrected(o, 0, n_tok, sel(q), sel(kr), sel(vr), T.sigma_of(128))
-    for kname, kflag in (("tcgen05", B.KVQ_KERNEL_TCGEN05), ("mma_sync", B.KVQ_KERNEL_MMA_SYNC)):
+    for kname, kflag in (("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR), ("mma_sync", B.KVQ_KERNEL_MMA_SYNC)):
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         out = B.kvq_attn_corrected(g, T.to_dev(q), T.to_dev(kr), T.to_dev(vr), T.sigma_of(128),
                                    B.KVQ_CORRECTION_ON | kflag, cache_begin=begin, cache_len=n_tok, status_word=status)

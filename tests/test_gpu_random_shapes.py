@@ -54,7 +54,7 @@ def test_random_shape(c):
     begin = start + c["begin"]
     want = O.attn_corrected(o, begin, c["n_cached"], q, kc, vc, sigma, correction=c["corr"])
     flag = B.KVQ_CORRECTION_ON if c["corr"] else B.KVQ_CORRECTION_OFF
-    for kname, kflag in [("mma_sync", B.KVQ_KERNEL_MMA_SYNC)] + ([("tcgen05", B.KVQ_KERNEL_TCGEN05)] if d == 128 else []):
+    for kname, kflag in [("mma_sync", B.KVQ_KERNEL_MMA_SYNC)] + ([("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR)] if d == 128 else []):
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         lse = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
         mass = torch.zeros_like(lse)

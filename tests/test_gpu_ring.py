@@ -54,7 +54,7 @@ def test_attention_over_a_wrapping_window(B, d):
         begin -= begin % 16                                         # window starts are multiples of 16 tokens
         length = min(length, n - begin)
         want = O.attn_corrected(o, begin, length, q, kc, vc, T.sigma_of(d))
-        for kname, kflag in ([("mma_sync", B.KVQ_KERNEL_MMA_SYNC)] + ([("tcgen05", B.KVQ_KERNEL_TCGEN05)] if d == 128 else [])):
+        for kname, kflag in ([("mma_sync", B.KVQ_KERNEL_MMA_SYNC)] + ([("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR)] if d == 128 else [])):
             status = torch.zeros(1, dtype=torch.int32, device="cuda")
             mass = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")
             out = B.kvq_attn_corrected(g, qd, kd, vd, T.sigma_of(d), B.KVQ_CORRECTION_ON | kflag, cache_begin=begin,

@@ -39,7 +39,7 @@ def test_rotated_values_append_and_attention(B, d, bits, group, with_signs):
     for name in ("k_codes", "v_codes", "k_scale", "v_scale", "k_zero", "v_zero"):
         getattr(plain, name)[:] = getattr(o, name)
     assert np.abs(O.attn_corrected(plain, 0, n, q, kc, vc, sigma)["out"] - want["out"]).max() > 0.1   # the flag matters
-    kernels = [("mma_sync", B.KVQ_KERNEL_MMA_SYNC)] + ([("tcgen05", B.KVQ_KERNEL_TCGEN05)] if d == 128 else [])
+    kernels = [("mma_sync", B.KVQ_KERNEL_MMA_SYNC)] + ([("tcgen05", B.KVQ_KERNEL_TCGEN05), ("tcgen05_pair", B.KVQ_KERNEL_TCGEN05_PAIR)] if d == 128 else [])
     for kname, kflag in kernels:
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         mass = torch.zeros(q.shape[:3], dtype=torch.float32, device="cuda")

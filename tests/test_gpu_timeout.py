@@ -15,7 +15,8 @@ pytestmark = pytest.mark.gpu
 SITE_CODES = {100, 101, 102, 103, 201, 203, 204, 205, 207, 209, 301, 302, 303, 401, 402, 404}
 
 
-def test_expired_wait_sets_the_status_word_and_the_kernel_returns():
+@pytest.mark.parametrize("kernel", ["KVQ_KERNEL_TCGEN05", "KVQ_KERNEL_TCGEN05_PAIR"])
+def test_expired_wait_sets_the_status_word_and_the_kernel_returns(kernel):
     from paper_2605_26266_b200 import binding as B
     w = inputs.Workload("timeout", 91, 1, 1, 128, 256, 2, 2, 128, 3)     # one unit of 256 rows: one CTA, 6 key tiles
     g = B.Cache(w.batch, w.heads, w.head_dim, w.bits, w.group, w.capacity)
@@ -28,7 +29,7 @@ def test_expired_wait_sets_the_status_word_and_the_kernel_returns():
     q, k, v = inputs.make_chunk(w, w.cached_chunks)
     qd, kd, vd = T.to_dev(q), T.to_dev(k), T.to_dev(v)
     sigma = T.sigma_of(w.head_dim)
-    flags = B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05
+    flags = B.KVQ_CORRECTION_ON | getattr(B, kernel)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     try:
         B.kvq_set_wait_budget_cycles(2)
