@@ -204,6 +204,27 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Of every four pairs of scores, how many take their exponentials on the FMA pipe instead of the MUFU (16 lanes
+// per SM: the two softmax warps of a scheduler share 4).  Measured: one of four is worth 2 to 5 % in the pair
+// kernel, where the MUFU is what the softmax groups wait for; in the one-CTA kernel the extra instructions cost as
+// much as they save, so it keeps the MUFU for all.
+constexpr int kPolyPairs = 1;
+// 2^x for a pair of arguments without the MUFU: x = n + r with n the nearest integer (taken from the low mantissa
+// bits of x + 1.5 * 2^23) and r in [-0.5, 0.5]; 2^r by a cubic (relative error 7.5e-5, far below the BF16
+// rounding that follows); n goes into the exponent field by an integer add.  Arguments are clamped at -125, so
+// the result is at least 2^-126 where the MUFU would flush to zero; x may be -inf.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  const float kMagic = 12582912.f;
+  x.x = fmaxf(x.x, -125.f); x.y = fmaxf(x.y, -125.f);
+  const float2 fl = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(fl, make_float2(-kMagic, -kMagic));
+  const float2 r = __fadd2_rn(x, make_float2(-n.x, -n.y));
+  float2 q = __ffma2_rn(r, make_float2(0.05517164617776871f, 0.05517164617776871f), make_float2(0.2426111251115799f, 0.2426111251115799f));
+  q = __ffma2_rn(q, r, make_float2(0.6932609677314758f, 0.6932609677314758f));
+  q = __ffma2_rn(q, r, make_float2(0.9999280571937561f, 0.9999280571937561f));
+  return make_float2(__uint_as_float(__float_as_uint(q.x) + (__float_as_uint(fl.x) << 23)),
+                     __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(fl.y) << 23)));
+}
 __device__ __forceinline__ uint32_t hfma2_f16(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t d;
   asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -879,7 +900,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int i = 0; i < 64; i += 2) {
             const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), c2, nm2);
-            const float2 pr = make_float2(ex2(x.x), ex2(x.y));
+            const float2 pr = ((i >> 1) & 3) < (PAIR ? kPolyPairs : 0) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
             sum2 = __fadd2_rn(sum2, pr);
             sr[i >> 1] = cvt_bf16x2(pr.x, pr.y);
           }
@@ -1204,8 +1225,8 @@ int num_sms() {
 
 // Grid policy: how many CTAs, and how many leading units are computed whole (the rest are split).
 //  * At least as many units as SMs: one persistent CTA per SM.  Whole units are dealt out in rounds of
-//    one per CTA; the last, incomplete round of R units would leave SMs idle for a whole unit's time, so
-//    when R is at most half the SMs its key-tile steps are split evenly over all CTAs instead.
+//    one per CTA; the last, incomplete round of R units would leave sms - R SMs idle for a whole unit's
+//    time, so its key-tile steps are split evenly over all CTAs instead, when that is worth its cost (below).
 //  * Fewer units than SMs: one CTA per unit leaves sms - n_units SMs idle for `tiles` tile steps each.
 //    Cutting all tile steps into equal ranges, one per SM, uses them, at a measured cost of about ten
 //    tile steps per CTA (a second prologue and epilogue, FP32 partial results, the merge kernel): split
@@ -1215,7 +1236,7 @@ Plan plan_grid(int64_t n_units, int64_t tiles, bool pair = false) {
   const int sms = pair ? num_sms() / 2 : num_sms();      // CTAs, or CTA pairs, that run at once
   if (n_units >= sms) {
     const int64_t r = n_units % sms;
-    return {sms, (int)((r == 0 || 2 * r > sms) ? n_units : n_units - r)};
+    return {sms, (int)((r == 0 || tiles * (sms - r) <= 10 * (int64_t)sms) ? n_units : n_units - r)};
   }
   if (tiles * (sms - n_units) <= 10 * (int64_t)sms) return {(int)n_units, (int)n_units};
   const int64_t W = n_units * tiles;

@@ -100,7 +100,14 @@ static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur
   if ((kern == KVQ_KERNEL_TCGEN05 || kern == KVQ_KERNEL_TCGEN05_PAIR) && !ok) *err = KVQ_ERR_UNSUPPORTED;
   return ok;
 }
-static bool is_pair(uint32_t flags) { return (flags & KVQ_KERNEL_MASK) == KVQ_KERNEL_TCGEN05_PAIR; }
+// Which tcgen05 kernel: the one asked for, else (KVQ_KERNEL_AUTO) the pair kernel unless its units of 512 query
+// rows pad the chunk so much more than units of 256 that its measured advantage per row (12 % or more) is lost.
+static bool is_pair(uint32_t flags, int64_t m_tokens) {
+  const uint32_t kern = flags & KVQ_KERNEL_MASK;
+  if (kern != KVQ_KERNEL_AUTO) return kern == KVQ_KERNEL_TCGEN05_PAIR;
+  const int64_t rows_pair = (m_tokens + 511) / 512 * 512, rows_single = (m_tokens + 255) / 256 * 256;
+  return rows_pair * 88 <= rows_single * 100;
+}
 
 // Checks shared by the two attention entry points, then the argument block the launchers take.
 static int check_attn_call(const kvq_cache_desc* d, int64_t cache_begin, int64_t cache_len, const void* q,
@@ -198,7 +205,7 @@ int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags)) : 0);
+  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags, m_tokens)) : 0);
   return KVQ_OK;
 }
 
@@ -210,7 +217,7 @@ int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur, is_pair(flags)) : (m_tokens > 0 ? 1 : 0)) +
+  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur, is_pair(flags, m_tokens)) : (m_tokens > 0 ? 1 : 0)) +
                (rotv_bytes(desc, cache_len, m_tokens, n_cur) ? 2 : 0);      // value pre-pass and output post-pass
   return KVQ_OK;
 }
@@ -238,13 +245,15 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   }
   const size_t rotv = rotv_bytes(desc, cache_len, m_tokens, n_cur);
   {
-    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags)) : 0);
+    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags, m_tokens)) : 0);
     if (need > 0) {
       if (!workspace || workspace_bytes < need) return KVQ_ERR_WORKSPACE;
       if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return KVQ_ERR_ALIGNMENT;
     }
   }
   if (m_tokens == 0) return KVQ_OK;
+  if (tc)     // the launcher takes the choice between the two tcgen05 kernels from the flags
+    a.flags = (a.flags & ~KVQ_KERNEL_MASK) | (is_pair(flags, m_tokens) ? KVQ_KERNEL_TCGEN05_PAIR : KVQ_KERNEL_TCGEN05);
   if (rotv) {
     // values are cached rotated: bring the current chunk's values into the same space, attend, rotate the output back
     const kvq_strides dense{(int64_t)desc->heads * n_cur * desc->head_dim, n_cur * (int64_t)desc->head_dim, (int64_t)desc->head_dim};
