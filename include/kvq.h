@@ -81,12 +81,16 @@ extern "C" {
                                       KVQ_CORRECTION_ON.  Warp-level kernel only (KVQ_KERNEL_AUTO picks it;
                                       KVQ_KERNEL_TCGEN05 and the static-scratch entry return
                                       KVQ_ERR_UNSUPPORTED): an analysis option, several times slower. */
-#define KVQ_KERNEL_AUTO       0u
+#define KVQ_KERNEL_AUTO       0u         /* head_dim 128 with TMA-addressable strides: the pair kernel unless its units of 512
+                                            query rows pad m_tokens too far beyond a multiple of 256, then the one-CTA
+                                            tcgen05 kernel; everything else: the warp-level kernel */
 #define KVQ_KERNEL_MMA_SYNC   (1u << 8)  /* force the warp-level mma.sync kernel (cross-check / fallback shapes) */
 #define KVQ_KERNEL_TCGEN05    (2u << 8)  /* force the tcgen05/TMEM kernel; KVQ_ERR_UNSUPPORTED if the shape is not covered */
 #define KVQ_KERNEL_TCGEN05_PAIR (3u << 8) /* the tcgen05 kernel on pairs of SMs (thread-block clusters of two CTAs that share
                                             one tcgen05.mma of 256 rows): each CTA of a pair expands only half of every
-                                            cached key and value tile.  Same results; same shapes as KVQ_KERNEL_TCGEN05 */
+                                            cached key and value tile.  Same shapes as KVQ_KERNEL_TCGEN05; results equal to
+                                            its within rounding (a quarter of the exponentials are a cubic on the FMA
+                                            pipe, relative error 7.5e-5, before the BF16 rounding of the weights) */
 #define KVQ_KERNEL_MASK       (3u << 8)
 
 typedef void* kvq_stream_t;          /* a cudaStream_t */
