@@ -1231,9 +1231,37 @@ int num_sms() {
 //    Cutting all tile steps into equal ranges, one per SM, uses them, at a measured cost of about ten
 //    tile steps per CTA (a second prologue and epilogue, FP32 partial results, the merge kernel): split
 //    when the idle time is worth more than that.
+// CTA pairs that can be resident at once on the current device: a cluster of two needs two free SMs of one GPC,
+// so a device whose GPCs hold odd numbers of usable SMs fits fewer pairs than SMs / 2, and a persistent grid
+// larger than that would run its last clusters after all the others.  Asked once per device; SMs / 2 if the
+// device cannot be asked (the launch then fails loudly by itself).
+int max_resident_pairs() {
+  static std::atomic<int> cache[kMaxDevices] = {};
+  int dev = 0;
+  if (current_device(&dev) != KVQ_OK) return num_sms() / 2;
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    auto kern = attn_tcgen05_kernel<2, 128, true>;     // every instantiation has the same footprint
+    n = num_sms() / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)n); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess &&
+        cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) == cudaSuccess && clusters > 0 && clusters < n)
+      n = clusters;
+    (void)cudaGetLastError();
+    cache[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+
 struct Plan { int ctas; int n_whole; };
 Plan plan_grid(int64_t n_units, int64_t tiles, bool pair = false) {
-  const int sms = pair ? num_sms() / 2 : num_sms();      // CTAs, or CTA pairs, that run at once
+  const int sms = pair ? max_resident_pairs() : num_sms();      // CTAs, or CTA pairs, that run at once
   if (n_units >= sms) {
     const int64_t r = n_units % sms;
     return {sms, (int)((r == 0 || tiles * (sms - r) <= 10 * (int64_t)sms) ? n_units : n_units - r)};
