@@ -82,8 +82,9 @@ extern "C" {
                                       KVQ_KERNEL_TCGEN05 and the static-scratch entry return
                                       KVQ_ERR_UNSUPPORTED): an analysis option, several times slower. */
 #define KVQ_KERNEL_AUTO       0u         /* head_dim 128 with TMA-addressable strides: the pair kernel unless its units of 512
-                                            query rows pad m_tokens too far beyond a multiple of 256, then the one-CTA
-                                            tcgen05 kernel; everything else: the warp-level kernel */
+                                            query rows pad m_tokens too far beyond a multiple of 256 (by more than 1/0.88
+                                            at 2 bits, 1/0.86 at 4), then the one-CTA tcgen05 kernel; everything else: the
+                                            warp-level kernel */
 #define KVQ_KERNEL_MMA_SYNC   (1u << 8)  /* force the warp-level mma.sync kernel (cross-check / fallback shapes) */
 #define KVQ_KERNEL_TCGEN05    (2u << 8)  /* force the tcgen05/TMEM kernel; KVQ_ERR_UNSUPPORTED if the shape is not covered */
 #define KVQ_KERNEL_TCGEN05_PAIR (3u << 8) /* the tcgen05 kernel on pairs of SMs (thread-block clusters of two CTAs that share
@@ -280,10 +281,10 @@ int kvq_unpack_codes(const kvq_cache_desc* desc, int which, int64_t begin, int64
  * CTA, every role of that CTA leaves its loop at its next wait, work in flight is drained, and the kernel
  * returns.  The first site code reaches the caller's status_word; the outputs are then undefined.
  * Site codes: TMA producer 100 (query buffer free), 101 (key stage free), 102 (value stage free), 103 (last
- * unrotated score product done); MMA issuer 201 (query tile), 203 (value tile), 204 (probabilities), 205 (key
+ * unrotated score product done), 104 (stage of the packed-tile ring free); MMA issuer 201 (query tile), 203 (value tile), 204 (probabilities), 205 (key
  * tile), 207 (rotated query), 209 (output accumulator read out); softmax warps 301 (scores), 302 (product
  * retired before a rescale), 303 (last product before the epilogue); dequantization warps 401 (key stage free),
- * 402 (query tile, for the bias rows), 404 (value stage free).
+ * 402 (query tile, for the bias rows), 404 (value stage free), 406 (packed tile in the ring).
  *
  * kvq_status_word_result maps a status word read back by the caller (host value) to KVQ_OK (0) or
  * KVQ_ERR_TIMEOUT (anything else).

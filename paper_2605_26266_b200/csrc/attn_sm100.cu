@@ -68,7 +68,7 @@ constexpr int kOffV = kOffK + 2 * kTileBytes;      // 2 stages
 constexpr int kOffAx = kOffV + 2 * kTileBytes;     // 2 query tiles
 constexpr int kOffBx = kOffAx + 2 * kXBytes;       // 2 stages
 constexpr int kOffBar = kOffBx + 2 * kXBytes;
-constexpr int kNumBars = 28;                       // mbarriers, 8 bytes each (enum Bar below)
+constexpr int kNumBars = 32;                       // mbarriers, 8 bytes each (enum Bar below)
 static_assert(kNumBars * 8 <= 256, "barrier area");
 constexpr int kOffMisc = kOffBar + 256;
 constexpr int kSmemBytes = kOffMisc + 64 + 1024;   // + slack to align the base to 1024
@@ -76,7 +76,21 @@ constexpr int kSmemBytes = kOffMisc + 64 + 1024;   // + slack to align the base 
 // kSFull, kPFull and kODone have four barriers each: index 2 * (half of the key tile) + (query tile); each of
 // them completes once per key tile, so that a waiter is never more than one phase behind
 enum Bar { kQFull = 0, kKFull = 1, kVFull = 3, kKEmpty = 5, kVEmpty = 7, kSFull = 9, kPFull = 13,
-           kODone = 17, kQCurDone = 21, kQRotFull = 22, kDrain = 23, kQEmpty = 25, kOFree = 26 };
+           kODone = 17, kQCurDone = 21, kQRotFull = 22, kDrain = 23, kQEmpty = 25, kOFree = 26,
+           kRawFull = 28, kRawEmpty = 30 };
+
+// Pair kernel only: a CTA of a pair fills half of every operand stage (64 of the 128 key rows of each 64-column
+// block, one of the two 64-channel value blocks), and the other half holds the staging ring for the PACKED tiles:
+// codes and metadata of the 128 cached tokens of a tile, brought in by bulk copies one tile ahead, two stages.
+// Codes of stage r sit in the unused value block of operand stage r (keys' codes, then values' codes, 8 KiB
+// each), metadata in the unused rows of its first key block (key scales, key zero-points, value scales, value
+// zero-points).
+constexpr int kRawCodesOff = kHalfTile;            // from the start of the value stage
+constexpr int kRawVCodes = 8192;                   // values' codes after the keys' codes
+constexpr int kRawMetaOff = 64 * 128;              // from the start of the key stage: behind its 64 rows in use
+constexpr int kRawKZero = 512, kRawVScale = 1536, kRawVZero = 2048;
+static_assert(128 * (kD * 4 / 8) <= kRawVCodes && 2 * kRawVCodes <= kHalfTile, "packed codes fit the unused value block");
+static_assert(kRawVZero + 128 * 4 * 2 <= kHalfTile - kRawMetaOff, "metadata fits the unused key rows");
 
 constexpr uint32_t kTimeoutCycles = 2000000000u;   // about a second; 32-bit clock differences stay exact below 2^32
 constexpr uint32_t kDrainCycles = 20000000u;
@@ -291,6 +305,34 @@ __device__ __forceinline__ void load_raw(Raw<BITS>& r, const uint8_t* codes, con
   } else {
     r.sbytes = __ldg(reinterpret_cast<const uint32_t*>(scale + tok * 4));
     const uint2 z = __ldg(reinterpret_cast<const uint2*>(zero + tok * 4));
+    r.z01 = z.x; r.z23 = z.y;
+  }
+}
+
+// The same from the staging ring in shared memory (pair kernel): `key` is the token's place in its tile.
+template <int BITS, int G, int NW>
+__device__ __forceinline__ void load_raw_staged(Raw<BITS>& r, const uint8_t* codes, const uint8_t* scale, const uint8_t* zero,
+                                                int key, bool valid, int word0) {
+  if (!valid) {
+#pragma unroll
+    for (int i = 0; i < NW; ++i) r.w[i] = 0;
+    r.sbytes = 0; r.z01 = 0; r.z23 = 0;
+    return;
+  }
+  const uint4* cw = reinterpret_cast<const uint4*>(codes + key * (kD * BITS / 8)) + (word0 >> 2);
+#pragma unroll
+  for (int i = 0; i < NW / 4; ++i) {
+    const uint4 v = cw[i];
+    r.w[4 * i] = v.x; r.w[4 * i + 1] = v.y; r.w[4 * i + 2] = v.z; r.w[4 * i + 3] = v.w;
+  }
+  if constexpr (G == 1) {
+    r.sbytes = scale[key]; r.z01 = *reinterpret_cast<const uint16_t*>(zero + key * 2); r.z23 = 0;
+  } else if constexpr (G == 2) {
+    r.sbytes = *reinterpret_cast<const uint16_t*>(scale + key * 2);
+    r.z01 = *reinterpret_cast<const uint32_t*>(zero + key * 4); r.z23 = 0;
+  } else {
+    r.sbytes = *reinterpret_cast<const uint32_t*>(scale + key * 4);
+    const uint2 z = *reinterpret_cast<const uint2*>(zero + key * 8);
     r.z01 = z.x; r.z23 = z.y;
   }
 }
@@ -527,7 +569,10 @@ __global__ void __launch_bounds__(256) rotate_query_kernel(const RotParams p) {
 // dequantization work, the stores and the B-operand reads per SM halve.  The leader CTA (rank 0) issues every
 // MMA, with M = 256: 128 rows in each CTA's own TMEM.  Barriers the issuer waits on live in the leader and take
 // arrivals from both CTAs; barriers the issuer signals are committed to both CTAs at once.  No load is multicast:
-// each CTA fetches its own half.
+// each CTA fetches its own half.  The halves of the operand stages a CTA of a pair does not use hold a two-stage
+// ring for the PACKED tiles: the TMA thread brings the codes and metadata of the next cached tile in with bulk
+// copies, and the dequant warps expand them from shared memory (the one-CTA kernel has no room for that and
+// reads them from global memory into registers a tile ahead).
 template <int BITS, int GROUP, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qr,
@@ -577,6 +622,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(cx.bar(kDrain + 0), 1);
     mbar_init(cx.bar(kDrain + 1), 1);
     mbar_init(cx.bar(kQEmpty), 2);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(cx.bar(kRawFull + s), 1);     // the TMA thread's expect-tx; the copies complete the bytes
+      mbar_init(cx.bar(kRawEmpty + s), 128);  // the dequant threads have the stage's contents in registers
+    }
     mbar_init(cx.bar(kOFree + 0), 128 * kC);
     mbar_init(cx.bar(kOFree + 1), 128 * kC);
     fence_barrier_init();
@@ -606,6 +655,36 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if constexpr (PAIR) tma_load_4d_pair(dst, map, bar, c0, c1, c2, c3);
         else tma_load_4d(dst, map, bar, c0, c1, c2, c3);
       };
+      // Pair kernel: the packed codes and metadata of cached tile ct of (batch, head) bh into the next stage of
+      // the staging ring.  A tile is 128 consecutive slots of the head's slab, taken modulo the capacity: one run,
+      // or two where the window wraps.  Slot numbers are multiples of 16 (cache_begin is, the capacity is a
+      // multiple of 128), so every source address and size below is a multiple of 16 bytes.
+      int n_raw = 0;
+      auto stage_packed = [&](int ct, int bh) -> bool {
+        constexpr int kCB = kD * BITS / 8;
+        const int rs = n_raw & 1;
+        if (!cx.wait(kRawEmpty + rs, ((n_raw >> 1) & 1) ^ 1, 104)) return false;
+        const uint32_t bar = cx.bar(kRawFull + rs);
+        mbar_arrive_expect_tx(bar, 128u * (2 * kCB + 6 * G));
+        const uint32_t codes = sbase + kOffV + rs * kTileBytes + kRawCodesOff;
+        const uint32_t meta = sbase + kOffK + rs * kTileBytes + kRawMetaOff;
+        int64_t slot = p.cache_begin + (int64_t)ct * kBlockN;
+        if (slot >= p.capacity) slot -= p.capacity;
+        const int n1 = (int)min((int64_t)kBlockN, p.capacity - slot);
+        for (int part = 0; part < 2; ++part) {
+          const int n = part == 0 ? n1 : kBlockN - n1, at = part == 0 ? 0 : n1;
+          if (n == 0) break;
+          const int64_t tok = (int64_t)bh * p.capacity + (part == 0 ? slot : 0);
+          bulk_load(codes + at * kCB, p.k_codes + tok * kCB, n * kCB, bar);
+          bulk_load(codes + kRawVCodes + at * kCB, p.v_codes + tok * kCB, n * kCB, bar);
+          bulk_load(meta + at * G, p.k_scale + tok * G, n * G, bar);
+          bulk_load(meta + kRawKZero + at * 2 * G, p.k_zero + tok * G, n * 2 * G, bar);
+          bulk_load(meta + kRawVScale + at * G, p.v_scale + tok * G, n * G, bar);
+          bulk_load(meta + kRawVZero + at * 2 * G, p.v_zero + tok * G, n * 2 * G, bar);
+        }
+        ++n_raw;
+        return true;
+      };
       Schedule sch(sched_id, n_sched, p);
       Segment sg;
       int it = 0, nseg = 0, issued_it = -1, rot_seg = -1;
@@ -613,6 +692,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       while (ok && sch.next(sg)) {
         const int bh = sg.unit / p.q_blocks, b = bh / p.heads, h = bh - b * p.heads;
         const int row0 = unit_row0(sg.unit, bh);
+        const int t_first_cached = max(sg.tb, n_rt);
+        if constexpr (PAIR) {       // the segment's first cached tile; every later one is staged a tile ahead
+          if (t_first_cached < sg.te && !(ok = stage_packed(t_first_cached - n_rt, bh))) break;
+        }
         // the query buffer is free once every score MMA of the previous segment has retired (the MMA warp says so
         // in its last iteration, before the last P V products)
         if (!(ok = cx.wait(kQEmpty, (nseg & 1) ^ 1, 100))) break;
@@ -664,11 +747,15 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           } else {
             arrive_lead(kVFull + s);
           }
+          if constexpr (PAIR) {
+            if (t + 1 < sg.te && t + 1 > t_first_cached && !(ok = stage_packed(t + 1 - n_rt, bh))) break;
+          }
         }
         ++nseg;
       }
       // drain: give loads already in flight a bounded time to land before the CTA exits (of a pair, the barriers
       // are the leader's and count both CTAs' bytes; the peer stays until the leader has come through, below)
+      if (*cx.abort && n_raw > 0) cx.drain(kRawFull + ((n_raw - 1) & 1), ((n_raw - 1) >> 1) & 1);   // this CTA's own copies
       if (*cx.abort && rank == 0) {
         if (nseg > 0) cx.drain(kQFull, (nseg - 1) & 1);
         if (rot_seg >= 0) cx.drain(kQRotFull, rot_seg & 1);
@@ -982,6 +1069,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     Schedule sch(sched_id, n_sched, p);
     Segment sg;
     int it = 0, nseg = 0;
+    int n_raw = 0;                         // cached tiles taken from the staging ring so far (pair kernel)
     bool ok = true;
     Raw<BITS> rk, rv;
     while (ok && sch.next(sg)) {
@@ -994,7 +1082,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         return slab0 + (slot >= p.capacity ? slot - p.capacity : slot);
       };
       const int t_rot = max(sg.tb, n_rt);          // first cached tile of the segment: the query is rotated there
-      if (sg.te > n_rt) {
+      if (!PAIR && sg.te > n_rt) {                 // one CTA: packed data comes one tile ahead into registers
         const int k0 = (t_rot - n_rt) * kBlockN + k_key, v0 = (t_rot - n_rt) * kBlockN + dt;
         load_raw<BITS, G, kNW>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k0), k0 < p.n_cached, k_word0);
         load_raw<BITS, G, kNW>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(v0), v0 < p.n_cached, v_word0);
@@ -1007,6 +1095,15 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kKEmpty + s, ph ^ 1, 401));
         if (!ok) break;
         KVQ_STAMP(22);
+        // pair: the tile's packed codes and metadata are in the staging ring (the TMA thread keeps it a tile ahead)
+        const uint8_t* raw_codes = smem + kOffV + (n_raw & 1) * kTileBytes + kRawCodesOff;
+        const uint8_t* raw_meta = smem + kOffK + (n_raw & 1) * kTileBytes + kRawMetaOff;
+        if (PAIR && ct >= 0) {
+          ok = __all_sync(0xFFFFFFFFu, cx.wait(kRawFull + (n_raw & 1), (n_raw >> 1) & 1, 406));
+          if (!ok) break;
+          load_raw_staged<BITS, G, kNW>(rk, raw_codes, raw_meta, raw_meta + kRawKZero, k_key,
+                                        ct * kBlockN + k_key < p.n_cached, k_word0);
+        }
         if (ct >= 0) {
           dequant_keys<BITS, GROUP, kNW>(rk, smem + kOffK + s * kTileBytes, k_row, k_word0);
           if (p.correction && k_word0 == 0) {   // B_extra row: step_j^2, exact in BF16
@@ -1016,7 +1113,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             *reinterpret_cast<uint4*>(smem + kOffBx + s * kXBytes + xtile_offset(k_row, 0)) = make_uint4(b01, b23, b01, b23);
           }
           fence_proxy_async_smem();
-          if (t + 1 < sg.te) load_raw<BITS, G, kNW>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k1), k1 < p.n_cached, k_word0);
+          if (!PAIR && t + 1 < sg.te) load_raw<BITS, G, kNW>(rk, p.k_codes, p.k_scale, p.k_zero, tok_of(k1), k1 < p.n_cached, k_word0);
         }
         arrive_lead(kKFull + s);
         KVQ_STAMP(20);
@@ -1042,10 +1139,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         ok = __all_sync(0xFFFFFFFFu, cx.wait(kVEmpty + s, ph ^ 1, 404));
         if (!ok) break;
         KVQ_STAMP(23);
+        if (PAIR && ct >= 0) {
+          load_raw_staged<BITS, G, kNW>(rv, raw_codes + kRawVCodes, raw_meta + kRawVScale, raw_meta + kRawVZero, dt,
+                                        ct * kBlockN + dt < p.n_cached, v_word0);
+          mbar_arrive(cx.bar(kRawEmpty + (n_raw & 1)));      // the stage's contents are in registers
+          ++n_raw;
+        }
         if (ct >= 0) {
           dequant_values<BITS, GROUP, kNW>(rv, smem + kOffV + s * kTileBytes, dt, v_word0, v_piece0);
           fence_proxy_async_smem();
-          if (t + 1 < sg.te) load_raw<BITS, G, kNW>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(v1), v1 < p.n_cached, v_word0);
+          if (!PAIR && t + 1 < sg.te) load_raw<BITS, G, kNW>(rv, p.v_codes, p.v_scale, p.v_zero, tok_of(v1), v1 < p.n_cached, v_word0);
         }
         arrive_lead(kVFull + s);
         KVQ_STAMP(21);

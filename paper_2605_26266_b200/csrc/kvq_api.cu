@@ -101,12 +101,14 @@ static bool use_tcgen05(const kvq_cache_desc* d, int64_t m_tokens, int64_t n_cur
   return ok;
 }
 // Which tcgen05 kernel: the one asked for, else (KVQ_KERNEL_AUTO) the pair kernel unless its units of 512 query
-// rows pad the chunk so much more than units of 256 that its measured advantage per row (12 % or more) is lost.
-static bool is_pair(uint32_t flags, int64_t m_tokens) {
+// rows pad the chunk so much more than units of 256 that its measured advantage per row is lost (12 % or more at
+// 2 bits; more at 4 bits, where there is more dequantization work to halve: M = 1560 pads to 2048 against 1792,
+// and the pair kernel measures 1 % slower at 2 bits, 3 % faster at 4).
+static bool is_pair(const kvq_cache_desc* d, uint32_t flags, int64_t m_tokens) {
   const uint32_t kern = flags & KVQ_KERNEL_MASK;
   if (kern != KVQ_KERNEL_AUTO) return kern == KVQ_KERNEL_TCGEN05_PAIR;
   const int64_t rows_pair = (m_tokens + 511) / 512 * 512, rows_single = (m_tokens + 255) / 256 * 256;
-  return rows_pair * 88 <= rows_single * 100;
+  return rows_pair * (d->bits == 4 ? 86 : 88) <= rows_single * 100;
 }
 
 // Checks shared by the two attention entry points, then the argument block the launchers take.
@@ -205,7 +207,7 @@ int kvq_attn_workspace_bytes(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags, m_tokens)) : 0);
+  *out_bytes = rotv_bytes(desc, cache_len, m_tokens, n_cur) + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(desc, flags, m_tokens)) : 0);
   return KVQ_OK;
 }
 
@@ -217,7 +219,7 @@ int kvq_attn_kernel_launches(const kvq_cache_desc* desc, int64_t cache_len, int6
   int err;
   const bool tc = use_tcgen05(desc, m_tokens, n_cur, flags, &err);
   if (err != KVQ_OK) return err;
-  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur, is_pair(flags, m_tokens)) : (m_tokens > 0 ? 1 : 0)) +
+  *out_count = (tc ? attn_tcgen05_kernel_launches(desc, cache_len, m_tokens, n_cur, is_pair(desc, flags, m_tokens)) : (m_tokens > 0 ? 1 : 0)) +
                (rotv_bytes(desc, cache_len, m_tokens, n_cur) ? 2 : 0);      // value pre-pass and output post-pass
   return KVQ_OK;
 }
@@ -245,7 +247,7 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   }
   const size_t rotv = rotv_bytes(desc, cache_len, m_tokens, n_cur);
   {
-    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(flags, m_tokens)) : 0);
+    const size_t need = rotv + (tc ? attn_tcgen05_workspace_bytes(desc, cache_len, m_tokens, n_cur, is_pair(desc, flags, m_tokens)) : 0);
     if (need > 0) {
       if (!workspace || workspace_bytes < need) return KVQ_ERR_WORKSPACE;
       if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return KVQ_ERR_ALIGNMENT;
@@ -253,7 +255,7 @@ int kvq_attn_corrected(const kvq_cache_desc* desc, int64_t cache_begin, int64_t 
   }
   if (m_tokens == 0) return KVQ_OK;
   if (tc)     // the launcher takes the choice between the two tcgen05 kernels from the flags
-    a.flags = (a.flags & ~KVQ_KERNEL_MASK) | (is_pair(flags, m_tokens) ? KVQ_KERNEL_TCGEN05_PAIR : KVQ_KERNEL_TCGEN05);
+    a.flags = (a.flags & ~KVQ_KERNEL_MASK) | (is_pair(desc, flags, m_tokens) ? KVQ_KERNEL_TCGEN05_PAIR : KVQ_KERNEL_TCGEN05);
   if (rotv) {
     // values are cached rotated: bring the current chunk's values into the same space, attend, rotate the output back
     const kvq_strides dense{(int64_t)desc->heads * n_cur * desc->head_dim, n_cur * (int64_t)desc->head_dim, (int64_t)desc->head_dim};

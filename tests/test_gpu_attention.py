@@ -184,13 +184,14 @@ def test_auto_dispatch_and_forced_kernel_errors(B):
             assert e.value.status == B.KVQ_ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("m,expect", [(140, "KVQ_KERNEL_TCGEN05"), (256, "KVQ_KERNEL_TCGEN05"), (300, "KVQ_KERNEL_TCGEN05_PAIR"),
-                                      (1560, "KVQ_KERNEL_TCGEN05"), (2048, "KVQ_KERNEL_TCGEN05_PAIR")])
-def test_auto_picks_the_pair_kernel_by_padded_rows(B, m, expect):
+@pytest.mark.parametrize("m,bits,expect", [(140, 2, "KVQ_KERNEL_TCGEN05"), (256, 2, "KVQ_KERNEL_TCGEN05"),
+                                           (300, 2, "KVQ_KERNEL_TCGEN05_PAIR"), (1560, 2, "KVQ_KERNEL_TCGEN05"),
+                                           (1560, 4, "KVQ_KERNEL_TCGEN05_PAIR"), (2048, 2, "KVQ_KERNEL_TCGEN05_PAIR")])
+def test_auto_picks_the_pair_kernel_by_padded_rows(B, m, bits, expect):
     """KVQ_KERNEL_AUTO on head_dim 128: the pair kernel unless its 512-row units pad the chunk too far beyond a
-    multiple of 256.  The two tcgen05 kernels differ in a quarter of their exponentials, so the bytes of the output
+    multiple of 256 (a little further at 4 bits).  The two tcgen05 kernels differ in a quarter of their exponentials, so the bytes of the output
     tell which one ran (and both are checked against the oracle elsewhere)."""
-    w = inputs.Workload("autopair", 77, 1, 2, 128, m, 1, 2, 64, 0)
+    w = inputs.Workload("autopair", 77, 1, 2, 128, m, 1, bits, 64, 0)
     g, o, n, sel = _build(B, w, 1, tokens=700, cap=768)
     q, kc, vc = inputs.make_chunk(w, 2)
     qd, kd, vd = T.to_dev(q), T.to_dev(kc), T.to_dev(vc)

@@ -12,7 +12,7 @@ from tests import kvq_testlib as T
 
 pytestmark = pytest.mark.gpu
 
-SITE_CODES = {100, 101, 102, 103, 201, 203, 204, 205, 207, 209, 301, 302, 303, 401, 402, 404}
+SITE_CODES = {100, 101, 102, 103, 104, 201, 203, 204, 205, 207, 209, 301, 302, 303, 401, 402, 404, 406}
 
 
 @pytest.mark.parametrize("kernel", ["KVQ_KERNEL_TCGEN05", "KVQ_KERNEL_TCGEN05_PAIR"])
