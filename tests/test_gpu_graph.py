@@ -13,8 +13,9 @@ from tests import kvq_testlib as T
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("kernel", ["KVQ_KERNEL_TCGEN05", "KVQ_KERNEL_TCGEN05_PAIR"])
 @pytest.mark.parametrize("heads,tokens", [(4, 600), (40, 1560)])   # units split over the SMs + merge / persistent rounds of whole units
-def test_step_replayed_from_a_graph_equals_the_eager_step(heads, tokens):
+def test_step_replayed_from_a_graph_equals_the_eager_step(heads, tokens, kernel):
     from paper_2605_26266_b200 import binding as B
     w = inputs.WORKLOADS["sweep_int2"]
     sigma = 1.0 / math.sqrt(w.head_dim)
@@ -29,7 +30,7 @@ def test_step_replayed_from_a_graph_equals_the_eager_step(heads, tokens):
         return cache
 
     q, k, v = chunks[2]
-    flags = B.KVQ_CORRECTION_ON | B.KVQ_KERNEL_TCGEN05
+    flags = B.KVQ_CORRECTION_ON | getattr(B, kernel)
 
     eager = fresh()
     n = eager.length
