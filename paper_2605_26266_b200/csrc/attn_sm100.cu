@@ -34,13 +34,17 @@
 // are therefore usually ready when it asks for them.
 //
 // The roles' loops are written to stay small (rolled over halves, query tiles and MMA groups): the SM's
-// instruction cache, and the GPC-level one behind it, bound this kernel before any pipe does.
+// instruction cache, and the GPC-level one behind it, bounded this kernel before any pipe did; what bounds it
+// now is the chain through a softmax group (score load, maximum, exponentials, store, hand-over).
 //
 // Work is cut into units (batch*head, 256-row query block) of `tiles` key tiles each.  Persistent CTAs take
 // whole units in rounds; where that would leave SMs idle (a short last round, or fewer units than SMs) the
 // unit x tile steps are divided evenly over one CTA per SM instead, a CTA walks its range segment by
 // segment, split units leave partial results (their own normalised rows, running max, row sums) in the
 // caller's workspace and a small kernel merges them.
+//
+// The same source also gives the pair kernel (template parameter PAIR): a cluster of two CTAs on 512 query rows
+// whose tensor cores work as one (tcgen05 cta_group::2), described at the kernel.
 //
 // Every wait on an mbarrier is bounded: on expiry the CTA records a diagnostic in the caller's status
 // word, all roles leave their loops, in-flight work is drained with a bounded wait, TMEM is freed and the
